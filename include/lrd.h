@@ -1,0 +1,179 @@
+/*
+ * lrd.h - C ABI of the B200 (sm_100a) library for the training step of low-rank
+ * decomposed layers.
+ *
+ * A dense layer weight W[N x K] (N outputs, K inputs) is replaced by two factors,
+ *     V[K x r]  (input side, applied first)   and   U[N x r]  (output side, applied second),
+ * so that the layer is two consecutive fully connected layers (paper, Section 2, Fig. 1):
+ *     Z[M x r] = X[M x K] V            Y[M x N] = Z U^T + 1 b^T .
+ * (The paper writes W in R^{C x S} with C inputs and S outputs and calls the input-side
+ * factor U' and the output-side factor V' (Eq. 2); this header uses the letters above.)
+ * A k x k convolution is replaced by its Tucker-2 form (Eq. 4): a 1x1 convolution A[C x r1],
+ * a k x k core G[r2][k][k][r1] and a 1x1 convolution Bm[S x r2].
+ *
+ * Conventions that hold for every entry point
+ *  - All matrices are row-major.  Leading dimensions are in elements; 0 means packed.
+ *  - Pointers named X, V, U, bias, Y, Z_save, dY, dX, dU, dV, dbias, A, G, Bm, Z1_save, Z2_save,
+ *    dA, dG, dB and `workspace` are DEVICE pointers owned by the caller.  The library allocates
+ *    no device memory, keeps no per-call device state, and never synchronises: all work is
+ *    enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default stream).
+ *  - `workspace` must hold at least lrd_*_workspace_bytes(...) bytes and be 256-byte aligned.
+ *    Its contents are scratch: undefined on return, nothing is carried between calls.
+ *  - Storage is fp32 or bf16 (lrd_dtype_t); products always accumulate in fp32.  Outputs and
+ *    gradients have the storage type of the tensor they belong to and are overwritten.
+ *  - Errors are return codes.  Arguments are checked on the host before anything is launched;
+ *    nothing aborts, asserts or traps.  Every wait inside a kernel is bounded; a wait that runs
+ *    out raises a device-side flag that lrd_check_device_status() reports as LRD_ERR_TIMEOUT.
+ *  - Ranks and sizes that do not meet the alignment needs of the tensor-core path (every
+ *    leading dimension a multiple of 8 elements and every base pointer 16-byte aligned, bf16)
+ *    are supported through a slower general path; they are not errors.
+ *  - Devices other than compute capability 10.x return LRD_ERR_ARCH.  There is no CPU path.
+ */
+#ifndef LRD_H_
+#define LRD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LRD_OK = 0,
+    LRD_ERR_INVALID_ARG = 1,  /* NULL where a pointer is required, non-positive size, bad enum, ld too small */
+    LRD_ERR_BAD_RANK = 2,     /* r < 1 or r > min(K, N); no multiple fits in lrd_rank_quantize */
+    LRD_ERR_ALIGNMENT = 3,    /* a base pointer is not aligned to its element size / workspace not 256-B aligned */
+    LRD_ERR_WORKSPACE = 4,    /* workspace NULL or too small */
+    LRD_ERR_UNSUPPORTED = 5,  /* convolution geometry other than k = 3, stride 1, pad 1 */
+    LRD_ERR_ARCH = 6,         /* current device is not sm_100 */
+    LRD_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
+    LRD_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out (see lrd_check_device_status) */
+} lrd_status_t;
+
+typedef enum { LRD_F32 = 0, LRD_BF16 = 1 } lrd_dtype_t;
+
+/* Which factor of a two-factor layer is frozen this step (Section 2.2, Algorithm 2). */
+typedef enum { LRD_FREEZE_NONE = 0, LRD_FREEZE_U = 1, LRD_FREEZE_V = 2 } lrd_freeze_t;
+
+/* Which group of a Tucker-2 layer is frozen: both 1x1 factors (A, Bm) or the core G. */
+typedef enum { LRD_TK_FREEZE_NONE = 0, LRD_TK_FREEZE_FACTORS = 1, LRD_TK_FREEZE_CORE = 2 } lrd_tucker_freeze_t;
+
+typedef enum { LRD_ROUND_UP = 0, LRD_ROUND_DOWN = 1, LRD_ROUND_NEAREST = 2 } lrd_round_t;
+
+/* Bits returned by lrd_linear_bwd_plan. */
+enum {
+    LRD_PLAN_DZ = 1, LRD_PLAN_DX = 2, LRD_PLAN_DU = 4, LRD_PLAN_DB = 8, LRD_PLAN_DV = 16,
+    LRD_PLAN_NEEDS_Z = 32, LRD_PLAN_NEEDS_X = 64
+};
+
+/* Execution path selector for lrd_set_path (testing and measurement). */
+typedef enum {
+    LRD_PATH_AUTO = 0,     /* library chooses */
+    LRD_PATH_GENERAL = 1,  /* fp32-FMA kernels for every shape and alignment */
+    LRD_PATH_UNFUSED = 2,  /* tensor-core GEMMs, rank-r intermediate through the workspace */
+    LRD_PATH_FUSED = 3     /* fused tensor-core chain where the shape allows, else UNFUSED */
+} lrd_path_t;
+
+typedef struct {
+    int64_t M, K, N, r;             /* tokens, inputs, outputs, rank */
+    int64_t ldx, ldv, ldu, ldy, ldz; /* leading dimensions of X/dX, V/dV, U/dU, Y/dY, Z_save; 0 = packed */
+    int32_t dtype;                  /* lrd_dtype_t of every tensor of the layer */
+} lrd_linear_desc_t;
+
+typedef struct {
+    int64_t B, H, W, C, S, r1, r2;  /* NHWC activations [B][H][W][C] -> [B][H][W][S] */
+    int64_t k, stride, pad;         /* only k = 3, stride = 1, pad = 1 */
+    int32_t dtype;
+} lrd_tucker2_desc_t;
+
+/* ---- host-only helpers (no device, no stream) ------------------------------------------ */
+
+/* Rank quantization (Section 2.1, "Rank Optimization": ranks whose dimensions suit the hardware,
+ * e.g. 257 -> 256).  Rounds r to a multiple of `multiple` (UP: ceiling, DOWN: floor, NEAREST: ties
+ * up), then clamps to [multiple, largest multiple <= min(K, N)].  Returns the rank, or the
+ * negated lrd_status_t (-LRD_ERR_INVALID_ARG for non-positive arguments or a bad mode,
+ * -LRD_ERR_BAD_RANK when no multiple fits below min(K, N)). */
+int64_t lrd_rank_quantize(int64_t r, int64_t multiple, lrd_round_t mode, int64_t K, int64_t N);
+
+/* Sequential freezing (Algorithm 2).  Two-factor layers: even epoch -> the first-applied
+ * sub-layer L_r(0) = V is frozen, odd epoch -> L_r(1) = U.  Tucker-2 layers: even epoch ->
+ * L_r(0), L_r(2) (the 1x1 factors) frozen, odd epoch -> L_r(1) (the core).  e < 0 is treated by
+ * its parity. */
+lrd_freeze_t lrd_freeze_for_epoch(int64_t e);
+lrd_tucker_freeze_t lrd_tucker_freeze_for_epoch(int64_t e);
+
+/* The products lrd_linear_bwd runs under a freeze mask (Section 2.2: a frozen sub-layer passes the
+ * gradient through but gets no weight gradient), as LRD_PLAN_* bits; 0 for a bad mask. */
+uint32_t lrd_linear_bwd_plan(lrd_freeze_t freeze);
+
+const char* lrd_status_string(lrd_status_t s);
+
+/* Process-wide choice of execution path (default LRD_PATH_AUTO).  Returns LRD_ERR_INVALID_ARG
+ * for an unknown value.  Not thread-safe against concurrent launches. */
+lrd_status_t lrd_set_path(lrd_path_t path);
+
+/* Synchronises the current device, then reports and clears the device-side timeout flag:
+ * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
+lrd_status_t lrd_check_device_status(void);
+
+/* Scratch bytes lrd_linear_fwd (is_bwd = 0) or lrd_linear_bwd (is_bwd = 1) needs for this layer and
+ * mask, for whichever path the library may take.  0 on a bad descriptor. */
+size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t freeze, int is_bwd);
+size_t lrd_tucker2_workspace_bytes(const lrd_tucker2_desc_t* desc, lrd_tucker_freeze_t freeze, int is_bwd);
+size_t lrd_dense_workspace_bytes(const lrd_linear_desc_t* desc, int is_bwd);
+
+/* ---- decomposed fully connected layer (Section 2, Fig. 1; freezing: Section 2.2) --------- */
+
+/* Forward: Z = X V, Y = Z U^T + bias.
+ *   X[M x K] (ldx), V[K x r] (ldv), U[N x r] (ldu), bias[N] or NULL, Y[M x N] (ldy) out.
+ *   Z_save[M x r] (ldz) out: the rank-r intermediate kept for dU.  Required (non-NULL) unless
+ *   freeze == LRD_FREEZE_U, in which case it must be NULL and Z is never written to memory the
+ *   caller sees.  In bf16, Z is rounded to bf16 once between the two products. */
+lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
+                            const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward: dZ = dY U, dX = dZ V^T always (dX = NULL skips the second product);
+ *   U not frozen: dU[N x r] = dY^T Z_save, dbias[N] = column sums of dY (dbias may be NULL);
+ *   V not frozen: dV[K x r] = X^T dZ.
+ * A frozen factor's weight-gradient product is never launched; if its gradient pointer (and, for
+ * U, dbias) is non-NULL it is filled with zeros.  X may be NULL when V is frozen, Z_save may be
+ * NULL when U is frozen; the gradient pointer of an unfrozen factor must be non-NULL. */
+lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                            const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                            lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- the undecomposed layer, for comparison (the "original layer" of Algorithm 1) -------- */
+
+/* Y = X W^T + bias with W[N x K] (leading dimension desc->ldv; desc->r, ldu, ldz ignored). */
+lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const void* W, const void* bias, void* Y,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* dX = dY W (NULL skips), dW = dY^T X, dbias = column sums of dY (NULL skips). */
+lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* W, void* dX,
+                           void* dW, void* dbias, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- Tucker-2 decomposed 3x3 convolution (Eq. 4, Fig. 1) -------------------------------- */
+
+/* Forward: Z1 = X A (1x1, C -> r1); Z2 = conv3x3(Z1, G) (cross-correlation, stride 1, zero pad 1,
+ * r1 -> r2); Y = Z2 Bm^T + bias (1x1, r2 -> S).  NHWC: X[B][H][W][C], Y[B][H][W][S]; A[C x r1],
+ * G[r2][3][3][r1], Bm[S x r2], bias[S] or NULL.
+ *   Z1_save[B][H][W][r1]: required unless freeze == LRD_TK_FREEZE_CORE (then must be NULL);
+ *   Z2_save[B][H][W][r2]: required unless freeze == LRD_TK_FREEZE_FACTORS (then must be NULL). */
+lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, const void* A, const void* G,
+                             const void* Bm, const void* bias, void* Y, void* Z1_save, void* Z2_save,
+                             lrd_tucker_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward: dZ2 = dY Bm; dZ1 = conv3x3^T(dZ2, G); dX = dZ1 A^T (NULL skips);
+ *   factors not frozen: dB[S x r2] = dY^T Z2_save, dA[C x r1] = X^T dZ1, dbias = column sums of dY;
+ *   core not frozen:    dG[o][kh][kw][i] = sum_p dZ2[p][o] Z1_save[p shifted by (kh-1, kw-1)][i].
+ * Frozen groups: product not launched, non-NULL gradient pointers are zero-filled. */
+lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, const void* X, const void* A,
+                             const void* G, const void* Bm, const void* Z1_save, const void* Z2_save, void* dX,
+                             void* dA, void* dG, void* dB, void* dbias, lrd_tucker_freeze_t freeze,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LRD_H_ */

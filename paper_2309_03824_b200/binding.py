@@ -1,0 +1,209 @@
+"""Thin ctypes binding of liblrd_b200.so: same names as include/lrd.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (or None); the binding passes their device pointers and the
+current CUDA stream.  There is no fallback: if the library is not built or cannot be loaded,
+importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblrd_b200.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2309_03824_b200.build`")
+_lib = C.CDLL(LIB_PATH)
+
+# enums -------------------------------------------------------------------------------------------
+(LRD_OK, LRD_ERR_INVALID_ARG, LRD_ERR_BAD_RANK, LRD_ERR_ALIGNMENT, LRD_ERR_WORKSPACE, LRD_ERR_UNSUPPORTED,
+ LRD_ERR_ARCH, LRD_ERR_CUDA, LRD_ERR_TIMEOUT) = range(9)
+LRD_F32, LRD_BF16 = 0, 1
+LRD_FREEZE_NONE, LRD_FREEZE_U, LRD_FREEZE_V = 0, 1, 2
+LRD_TK_FREEZE_NONE, LRD_TK_FREEZE_FACTORS, LRD_TK_FREEZE_CORE = 0, 1, 2
+LRD_ROUND_UP, LRD_ROUND_DOWN, LRD_ROUND_NEAREST = 0, 1, 2
+LRD_PLAN_DZ, LRD_PLAN_DX, LRD_PLAN_DU, LRD_PLAN_DB, LRD_PLAN_DV, LRD_PLAN_NEEDS_Z, LRD_PLAN_NEEDS_X = 1, 2, 4, 8, 16, 32, 64
+LRD_PATH_AUTO, LRD_PATH_GENERAL, LRD_PATH_UNFUSED, LRD_PATH_FUSED = 0, 1, 2, 3
+
+EXPORTS = [
+    "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
+    "lrd_status_string", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
+    "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd",
+]
+
+
+class lrd_linear_desc_t(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("M", "K", "N", "r", "ldx", "ldv", "ldu", "ldy", "ldz")] + [("dtype", C.c_int32)]
+
+
+class lrd_tucker2_desc_t(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("B", "H", "W", "C", "S", "r1", "r2", "k", "stride", "pad")] + [("dtype", C.c_int32)]
+
+
+_vp, _sz, _i64, _int = C.c_void_p, C.c_size_t, C.c_int64, C.c_int
+_lib.lrd_rank_quantize.restype = _i64
+_lib.lrd_rank_quantize.argtypes = [_i64, _i64, _int, _i64, _i64]
+_lib.lrd_freeze_for_epoch.restype = _int
+_lib.lrd_freeze_for_epoch.argtypes = [_i64]
+_lib.lrd_tucker_freeze_for_epoch.restype = _int
+_lib.lrd_tucker_freeze_for_epoch.argtypes = [_i64]
+_lib.lrd_linear_bwd_plan.restype = C.c_uint32
+_lib.lrd_linear_bwd_plan.argtypes = [_int]
+_lib.lrd_status_string.restype = C.c_char_p
+_lib.lrd_status_string.argtypes = [_int]
+_lib.lrd_set_path.restype = _int
+_lib.lrd_set_path.argtypes = [_int]
+_lib.lrd_check_device_status.restype = _int
+_lib.lrd_check_device_status.argtypes = []
+_lib.lrd_linear_workspace_bytes.restype = _sz
+_lib.lrd_linear_workspace_bytes.argtypes = [C.POINTER(lrd_linear_desc_t), _int, _int]
+_lib.lrd_dense_workspace_bytes.restype = _sz
+_lib.lrd_dense_workspace_bytes.argtypes = [C.POINTER(lrd_linear_desc_t), _int]
+_lib.lrd_tucker2_workspace_bytes.restype = _sz
+_lib.lrd_tucker2_workspace_bytes.argtypes = [C.POINTER(lrd_tucker2_desc_t), _int, _int]
+_lib.lrd_linear_fwd.restype = _int
+_lib.lrd_linear_fwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 6 + [_int, _vp, _sz, _vp]
+_lib.lrd_linear_bwd.restype = _int
+_lib.lrd_linear_bwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 9 + [_int, _vp, _sz, _vp]
+_lib.lrd_dense_fwd.restype = _int
+_lib.lrd_dense_fwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 4 + [_vp, _sz, _vp]
+_lib.lrd_dense_bwd.restype = _int
+_lib.lrd_dense_bwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 6 + [_vp, _sz, _vp]
+_lib.lrd_tucker2_fwd.restype = _int
+_lib.lrd_tucker2_fwd.argtypes = [C.POINTER(lrd_tucker2_desc_t)] + [_vp] * 8 + [_int, _vp, _sz, _vp]
+_lib.lrd_tucker2_bwd.restype = _int
+_lib.lrd_tucker2_bwd.argtypes = [C.POINTER(lrd_tucker2_desc_t)] + [_vp] * 12 + [_int, _vp, _sz, _vp]
+
+
+class LrdError(RuntimeError):
+    def __init__(self, status):
+        self.status = int(status)
+        super().__init__(f"lrd status {self.status}: {lrd_status_string(self.status)}")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is not None:
+        return C.c_void_p(int(stream))
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ws(workspace):
+    if workspace is None:
+        return None, 0
+    return C.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def _check(status):
+    if status != LRD_OK:
+        raise LrdError(status)
+
+
+def linear_desc(M, K, N, r, dtype, ldx=0, ldv=0, ldu=0, ldy=0, ldz=0):
+    return lrd_linear_desc_t(M, K, N, r, ldx, ldv, ldu, ldy, ldz, dtype)
+
+
+def tucker2_desc(B, H, W, Cin, S, r1, r2, dtype, k=3, stride=1, pad=1):
+    return lrd_tucker2_desc_t(B, H, W, Cin, S, r1, r2, k, stride, pad, dtype)
+
+
+# host-only helpers ---------------------------------------------------------------------------------
+def lrd_rank_quantize(r, multiple, mode, K, N):
+    return int(_lib.lrd_rank_quantize(r, multiple, mode, K, N))
+
+
+def lrd_freeze_for_epoch(e):
+    return int(_lib.lrd_freeze_for_epoch(e))
+
+
+def lrd_tucker_freeze_for_epoch(e):
+    return int(_lib.lrd_tucker_freeze_for_epoch(e))
+
+
+def lrd_linear_bwd_plan(freeze):
+    return int(_lib.lrd_linear_bwd_plan(freeze))
+
+
+def lrd_status_string(status):
+    return _lib.lrd_status_string(int(status)).decode()
+
+
+def lrd_set_path(path):
+    _check(_lib.lrd_set_path(path))
+
+
+def lrd_check_device_status():
+    return int(_lib.lrd_check_device_status())
+
+
+def lrd_linear_workspace_bytes(desc, freeze, is_bwd):
+    return int(_lib.lrd_linear_workspace_bytes(C.byref(desc), freeze, int(is_bwd)))
+
+
+def lrd_dense_workspace_bytes(desc, is_bwd):
+    return int(_lib.lrd_dense_workspace_bytes(C.byref(desc), int(is_bwd)))
+
+
+def lrd_tucker2_workspace_bytes(desc, freeze, is_bwd):
+    return int(_lib.lrd_tucker2_workspace_bytes(C.byref(desc), freeze, int(is_bwd)))
+
+
+# device entry points ---------------------------------------------------------------------------------
+def lrd_linear_fwd(desc, X, V, U, bias, Y, Z_save, freeze, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_linear_fwd(C.byref(desc), _ptr(X), _ptr(V), _ptr(U), _ptr(bias), _ptr(Y), _ptr(Z_save), freeze, w, n,
+                             _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_linear_bwd(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_linear_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(V), _ptr(U), _ptr(Z_save), _ptr(dX), _ptr(dU),
+                             _ptr(dV), _ptr(dbias), freeze, w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_dense_fwd(desc, X, W, bias, Y, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_dense_fwd(C.byref(desc), _ptr(X), _ptr(W), _ptr(bias), _ptr(Y), w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_dense_bwd(desc, dY, X, W, dX, dW, dbias, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_dense_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(W), _ptr(dX), _ptr(dW), _ptr(dbias), w, n,
+                            _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_tucker2_fwd(desc, X, A, G, Bm, bias, Y, Z1_save, Z2_save, freeze, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_tucker2_fwd(C.byref(desc), _ptr(X), _ptr(A), _ptr(G), _ptr(Bm), _ptr(bias), _ptr(Y), _ptr(Z1_save),
+                              _ptr(Z2_save), freeze, w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_tucker2_bwd(desc, dY, X, A, G, Bm, Z1_save, Z2_save, dX, dA, dG, dB, dbias, freeze, workspace, stream=None,
+                    check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_tucker2_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(A), _ptr(G), _ptr(Bm), _ptr(Z1_save),
+                              _ptr(Z2_save), _ptr(dX), _ptr(dA), _ptr(dG), _ptr(dB), _ptr(dbias), freeze, w, n,
+                              _stream(stream))
+    if check:
+        _check(st)
+    return st

@@ -1,0 +1,24 @@
+// Fused two-product chain  Out[M x N2] = (In[M x K1] P[K1 x r]) Q[N2 x r]^T (+ bias)  with the
+// rank-r intermediate T[M x r] kept on chip (tensor memory -> bf16 -> shared memory), written to
+// memory only when the caller asks for it (T_save).  The forward pass is the chain (X, V, U),
+// the backward data pass is the chain (dY, U, V).
+#pragma once
+#include "common.cuh"
+
+namespace lrd {
+
+struct ChainArgs {
+    int64_t M, K1, r, N2;
+    const void* In; int64_t ld_in;     // [M x K1]
+    const void* P; int64_t ldp;        // [K1 x r]
+    const void* Q; int64_t ldq;        // [N2 x r]
+    const void* bias;                  // [N2] or nullptr
+    void* Out; int64_t ld_out;         // [M x N2]
+    void* T_save; int64_t ldt;         // [M x r] or nullptr
+    lrd_dtype_t dtype;
+};
+
+bool chain_eligible(const ChainArgs& c);
+lrd_status_t chain_launch(const ChainArgs& c, cudaStream_t stream);
+
+}  // namespace lrd

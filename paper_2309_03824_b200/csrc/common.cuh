@@ -1,0 +1,44 @@
+// Shared host/device declarations of the library (internal).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lrd.h"
+
+namespace lrd {
+
+// Device address of the flag a bounded wait raises when it runs out (one word, zero = fine);
+// nullptr if the address cannot be obtained.  Read and cleared by lrd_check_device_status().
+unsigned int* device_timeout_flag();
+lrd_status_t read_and_clear_device_timeout(bool* raised);
+
+// One matrix product  C[M x N] = op(A) op(B) (+ bias over columns), fp32 accumulate.
+//   a_mn_major = false: A stored [M x K] (k contiguous);  true: A stored [K x M] (m contiguous)
+//   b_mn_major = false: B stored [N x K] (k contiguous);  true: B stored [K x N] (n contiguous)
+struct GemmArgs {
+    int64_t M, N, K;
+    const void* A; int64_t lda; bool a_mn_major;
+    const void* B; int64_t ldb; bool b_mn_major;
+    void* C; int64_t ldc;
+    const void* bias;          // [N] or nullptr, same dtype as C
+    lrd_dtype_t dtype;         // storage type of A, B, C, bias
+};
+
+inline size_t elem_size(int dtype) { return dtype == LRD_BF16 ? 2 : 4; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// General fp32-FMA path (any shape, any alignment).
+lrd_status_t simt_gemm(const GemmArgs& g, cudaStream_t stream);
+lrd_status_t simt_colsum(const void* A, int64_t lda, int64_t M, int64_t N, void* out, lrd_dtype_t dtype,
+                         cudaStream_t stream);
+
+// One product on the path chosen by `path` (an lrd_path_t): the tensor-core kernel when the
+// operands qualify, else the general kernel.
+lrd_status_t run_gemm(const GemmArgs& g, int path, bool allow_split, float* partials, size_t partial_bytes,
+                      cudaStream_t s);
+GemmArgs make_gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
+                   bool b_mn, void* C, int64_t ldc, const void* bias, lrd_dtype_t dt);
+lrd_status_t zero_fill(void* p, int64_t rows, int64_t cols, int64_t ld, lrd_dtype_t dt, cudaStream_t s);
+
+}  // namespace lrd

@@ -1,0 +1,119 @@
+// Tucker-2 decomposed 3x3 convolution (NHWC): 1x1 product, 3x3 core, 1x1 product, and the
+// backward pass through them under a freeze mask.
+#include "conv.cuh"
+
+#include "tc.cuh"
+
+namespace lrd {
+namespace {
+
+struct Tk {
+    int64_t B, H, W, C, S, r1, r2, P;
+    lrd_dtype_t dt;
+};
+
+Tk parse(const lrd_tucker2_desc_t* d) {
+    Tk t;
+    t.B = d->B; t.H = d->H; t.W = d->W; t.C = d->C; t.S = d->S; t.r1 = d->r1; t.r2 = d->r2;
+    t.P = d->B * d->H * d->W;
+    t.dt = (lrd_dtype_t)d->dtype;
+    return t;
+}
+
+size_t act_bytes(const Tk& t, int64_t ch) { return align_up((size_t)(t.P > 0 ? t.P : 1) * ch * elem_size(t.dt), 256); }
+
+size_t split_bytes(const Tk& t) {
+    if (t.dt != LRD_BF16 || t.P < 1) return 0;
+    const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P), b = tc_split_workspace_bytes(t.C, t.r1, t.P);
+    return a > b ? a : b;
+}
+
+#define LRD_TRY(expr)                          \
+    do {                                       \
+        lrd_status_t st__ = (expr);            \
+        if (st__ != LRD_OK) return st__;       \
+    } while (0)
+
+}  // namespace
+
+lrd_status_t tucker2_check(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t freeze) {
+    if (!d) return LRD_ERR_INVALID_ARG;
+    if (freeze != LRD_TK_FREEZE_NONE && freeze != LRD_TK_FREEZE_FACTORS && freeze != LRD_TK_FREEZE_CORE)
+        return LRD_ERR_INVALID_ARG;
+    if (d->B < 0 || d->H < 1 || d->W < 1 || d->C < 1 || d->S < 1) return LRD_ERR_INVALID_ARG;
+    if (d->dtype != LRD_F32 && d->dtype != LRD_BF16) return LRD_ERR_INVALID_ARG;
+    if (d->r1 < 1 || d->r2 < 1 || d->r1 > d->C || d->r2 > d->S) return LRD_ERR_BAD_RANK;
+    if (d->k != 3 || d->stride != 1 || d->pad != 1) return LRD_ERR_UNSUPPORTED;
+    if (d->H > 32767 || d->W > 32767) return LRD_ERR_UNSUPPORTED;
+    return LRD_OK;
+}
+
+size_t tucker2_workspace_bytes(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t freeze, int is_bwd) {
+    if (tucker2_check(d, freeze) != LRD_OK) return 0;
+    const Tk t = parse(d);
+    return act_bytes(t, t.r1) + act_bytes(t, t.r2) + (is_bwd ? split_bytes(t) : 0);
+}
+
+lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void* A, const void* G, const void* Bm,
+                         const void* bias, void* Y, void* Z1_save, void* Z2_save, lrd_tucker_freeze_t freeze,
+                         void* ws, size_t ws_bytes, int path, cudaStream_t s) {
+    (void)freeze; (void)ws_bytes;
+    const Tk t = parse(d);
+    if (t.P == 0) return LRD_OK;
+    void* Z1 = Z1_save ? Z1_save : ws;
+    void* Z2 = Z2_save ? Z2_save : (void*)((uint8_t*)ws + act_bytes(t, t.r1));
+    LRD_TRY(run_gemm(make_gemm(t.P, t.r1, t.C, X, t.C, false, A, t.r1, true, Z1, t.r1, nullptr, t.dt), path, false, nullptr, 0, s));
+    LRD_TRY(conv3x3_fwd(Z1, G, Z2, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    return run_gemm(make_gemm(t.P, t.S, t.r2, Z2, t.r2, false, Bm, t.r2, false, Y, t.S, bias, t.dt), path, false, nullptr, 0, s);
+}
+
+lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void* X, const void* A, const void* G,
+                         const void* Bm, const void* Z1_save, const void* Z2_save, void* dX, void* dA, void* dG,
+                         void* dB, void* dbias, lrd_tucker_freeze_t freeze, void* ws, size_t ws_bytes, int path,
+                         cudaStream_t s) {
+    const Tk t = parse(d);
+    const bool factors = freeze != LRD_TK_FREEZE_FACTORS, core = freeze != LRD_TK_FREEZE_CORE;
+    // frozen group: no product is launched; gradient buffers the caller passed read as zero
+    if (!factors || t.P == 0) {
+        LRD_TRY(zero_fill(dA, t.C, t.r1, t.r1, t.dt, s));
+        LRD_TRY(zero_fill(dB, t.S, t.r2, t.r2, t.dt, s));
+        LRD_TRY(zero_fill(dbias, 1, t.S, t.S, t.dt, s));
+    }
+    if (!core || t.P == 0) LRD_TRY(zero_fill(dG, t.r2, 9 * t.r1, 9 * t.r1, t.dt, s));
+    if (t.P == 0) return LRD_OK;
+
+    void* dZ1 = ws;
+    void* dZ2 = (uint8_t*)ws + act_bytes(t, t.r1);
+    float* partials = (float*)((uint8_t*)ws + act_bytes(t, t.r1) + act_bytes(t, t.r2));
+    const size_t pbytes = ws_bytes - act_bytes(t, t.r1) - act_bytes(t, t.r2);
+
+    LRD_TRY(run_gemm(make_gemm(t.P, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
+    if (dX || factors) LRD_TRY(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    if (dX) LRD_TRY(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
+    if (factors) {
+        LRD_TRY(run_gemm(make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt), path, true, partials, pbytes, s));
+        LRD_TRY(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, partials, pbytes, s));
+        if (dbias) LRD_TRY(simt_colsum(dY, t.S, t.P, t.S, dbias, t.dt, s));
+    }
+    if (core) LRD_TRY(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    return LRD_OK;
+}
+
+// Core convolution dispatch: the general kernels for now serve every shape.
+lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
+                         int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
+    (void)path;
+    return simt_conv3x3_fwd(in, G, out, B, H, W, ci, co, dt, s);
+}
+lrd_status_t conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W, int64_t ci,
+                              int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
+    (void)path;
+    return simt_conv3x3_bwd_data(dout, G, din, B, H, W, ci, co, dt, s);
+}
+lrd_status_t conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
+                                int64_t ci, int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
+    (void)path;
+    return simt_conv3x3_bwd_filter(dout, in, dG, B, H, W, ci, co, dt, s);
+}
+
+}  // namespace lrd

@@ -1,0 +1,36 @@
+// Tucker-2 decomposed 3x3 convolution: composition of 1x1 products and the r1 -> r2 core.
+#pragma once
+#include "common.cuh"
+
+namespace lrd {
+
+lrd_status_t tucker2_check(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t freeze);
+size_t tucker2_workspace_bytes(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t freeze, int is_bwd);
+lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void* A, const void* G, const void* Bm,
+                         const void* bias, void* Y, void* Z1_save, void* Z2_save, lrd_tucker_freeze_t freeze,
+                         void* ws, size_t ws_bytes, int path, cudaStream_t s);
+lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void* X, const void* A, const void* G,
+                         const void* Bm, const void* Z1_save, const void* Z2_save, void* dX, void* dA, void* dG,
+                         void* dB, void* dbias, lrd_tucker_freeze_t freeze, void* ws, size_t ws_bytes, int path,
+                         cudaStream_t s);
+
+// General-path 3x3 core (stride 1, zero pad 1), NHWC, any channel counts.
+//   fwd:        out[p][o] = sum_{kh,kw,i} in[p + (kh-1, kw-1)][i] G[o][kh][kw][i]
+//   bwd_data:   din[p][i] = sum_{kh,kw,o} dout[p - (kh-1, kw-1)][o] G[o][kh][kw][i]
+//   bwd_filter: dG[o][kh][kw][i] = sum_p dout[p][o] in[p + (kh-1, kw-1)][i]
+lrd_status_t simt_conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
+                              int64_t co, lrd_dtype_t dt, cudaStream_t s);
+lrd_status_t simt_conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W,
+                                   int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s);
+lrd_status_t simt_conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
+                                     int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s);
+
+// Path dispatch for the core (tensor-core kernel where the shape qualifies, else general).
+lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
+                         int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
+lrd_status_t conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W, int64_t ci,
+                              int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
+lrd_status_t conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
+                                int64_t ci, int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
+
+}  // namespace lrd

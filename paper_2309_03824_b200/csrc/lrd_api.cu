@@ -1,0 +1,342 @@
+// C-ABI entry points: argument checks, freeze-mask dispatch and path selection.  Every step of
+// the layer runs in this library's own kernels; nothing here falls back to the host.
+#include <cuda_runtime.h>
+
+#include <atomic>
+
+#include "chain.cuh"
+#include "common.cuh"
+#include "conv.cuh"
+#include "tc.cuh"
+
+using namespace lrd;
+
+namespace {
+
+std::atomic<int> g_path{LRD_PATH_AUTO};
+
+lrd_status_t check_arch() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LRD_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return LRD_ERR_CUDA;
+    return major == 10 ? LRD_OK : LRD_ERR_ARCH;
+}
+
+bool elem_aligned(const void* p, int dtype) { return ((uintptr_t)p % elem_size(dtype)) == 0; }
+
+struct Linear {
+    int64_t M, K, N, r, ldx, ldv, ldu, ldy, ldz;
+    lrd_dtype_t dt;
+};
+
+lrd_status_t parse_linear(const lrd_linear_desc_t* d, Linear* L, bool dense) {
+    if (!d) return LRD_ERR_INVALID_ARG;
+    if (d->M < 0 || d->K < 1 || d->N < 1) return LRD_ERR_INVALID_ARG;
+    if (d->dtype != LRD_F32 && d->dtype != LRD_BF16) return LRD_ERR_INVALID_ARG;
+    L->M = d->M; L->K = d->K; L->N = d->N; L->dt = (lrd_dtype_t)d->dtype;
+    if (dense) {
+        L->r = 0;
+        L->ldv = d->ldv ? d->ldv : d->K;
+        if (L->ldv < d->K) return LRD_ERR_INVALID_ARG;
+        L->ldu = L->ldz = 0;
+    } else {
+        if (d->r < 1 || d->r > (d->K < d->N ? d->K : d->N)) return LRD_ERR_BAD_RANK;
+        L->r = d->r;
+        L->ldv = d->ldv ? d->ldv : d->r;
+        L->ldu = d->ldu ? d->ldu : d->r;
+        L->ldz = d->ldz ? d->ldz : d->r;
+        if (L->ldv < d->r || L->ldu < d->r || L->ldz < d->r) return LRD_ERR_INVALID_ARG;
+    }
+    L->ldx = d->ldx ? d->ldx : d->K;
+    L->ldy = d->ldy ? d->ldy : d->N;
+    if (L->ldx < d->K || L->ldy < d->N) return LRD_ERR_INVALID_ARG;
+    return LRD_OK;
+}
+
+lrd_status_t check_ws(const void* ws, size_t have, size_t need) {
+    if (need == 0) return LRD_OK;
+    if (!ws || have < need) return LRD_ERR_WORKSPACE;
+    if ((uintptr_t)ws % 256) return LRD_ERR_ALIGNMENT;
+    return LRD_OK;
+}
+
+lrd_status_t run_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes, cudaStream_t s) {
+    return lrd::run_gemm(g, g_path.load(), allow_split, partials, partial_bytes, s);
+}
+GemmArgs gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
+              bool b_mn, void* C, int64_t ldc, const void* bias, lrd_dtype_t dt) {
+    return make_gemm(M, N, K, A, lda, a_mn, B, ldb, b_mn, C, ldc, bias, dt);
+}
+
+size_t linear_z_bytes(const Linear& L) { return align_up((size_t)(L.M > 0 ? L.M : 1) * L.r * elem_size(L.dt), 256); }
+
+size_t linear_split_bytes(const Linear& L) {
+    if (L.dt != LRD_BF16 || L.M < 1) return 0;
+    const size_t a = tc_split_workspace_bytes(L.N, L.r, L.M), b = tc_split_workspace_bytes(L.K, L.r, L.M);
+    return a > b ? a : b;
+}
+
+#define LRD_TRY(expr)                          \
+    do {                                       \
+        lrd_status_t st__ = (expr);            \
+        if (st__ != LRD_OK) return st__;       \
+    } while (0)
+
+}  // namespace
+
+namespace lrd {
+
+lrd_status_t run_gemm(const GemmArgs& g, int path, bool allow_split, float* partials, size_t partial_bytes,
+                      cudaStream_t s) {
+    if (g.M <= 0 || g.N <= 0) return LRD_OK;
+    if (path != LRD_PATH_GENERAL && tc_gemm_eligible(g)) return tc_gemm(g, allow_split, partials, partial_bytes, s);
+    return simt_gemm(g, s);
+}
+
+lrd_status_t zero_fill(void* p, int64_t rows, int64_t cols, int64_t ld, lrd_dtype_t dt, cudaStream_t s) {
+    if (!p || rows <= 0 || cols <= 0) return LRD_OK;
+    const size_t e = elem_size(dt);
+    return cudaMemset2DAsync(p, (size_t)ld * e, 0, (size_t)cols * e, (size_t)rows, s) == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+GemmArgs make_gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
+                   bool b_mn, void* C, int64_t ldc, const void* bias, lrd_dtype_t dt) {
+    GemmArgs g;
+    g.M = M; g.N = N; g.K = K; g.A = A; g.lda = lda; g.a_mn_major = a_mn; g.B = B; g.ldb = ldb; g.b_mn_major = b_mn;
+    g.C = C; g.ldc = ldc; g.bias = bias; g.dtype = dt;
+    return g;
+}
+
+}  // namespace lrd
+
+extern "C" {
+
+int64_t lrd_rank_quantize(int64_t r, int64_t multiple, lrd_round_t mode, int64_t K, int64_t N) {
+    if (r < 1 || multiple < 1 || K < 1 || N < 1) return -(int64_t)LRD_ERR_INVALID_ARG;
+    const int64_t lim = K < N ? K : N;
+    const int64_t cap = lim / multiple * multiple;
+    if (cap == 0) return -(int64_t)LRD_ERR_BAD_RANK;
+    int64_t q;
+    switch (mode) {
+        case LRD_ROUND_UP: q = (r + multiple - 1) / multiple * multiple; break;
+        case LRD_ROUND_DOWN: q = r / multiple * multiple; break;
+        case LRD_ROUND_NEAREST: q = (2 * r + multiple) / (2 * multiple) * multiple; break;
+        default: return -(int64_t)LRD_ERR_INVALID_ARG;
+    }
+    if (q < multiple) q = multiple;
+    if (q > cap) q = cap;
+    return q;
+}
+
+lrd_freeze_t lrd_freeze_for_epoch(int64_t e) { return (e % 2 == 0) ? LRD_FREEZE_V : LRD_FREEZE_U; }
+
+lrd_tucker_freeze_t lrd_tucker_freeze_for_epoch(int64_t e) {
+    return (e % 2 == 0) ? LRD_TK_FREEZE_FACTORS : LRD_TK_FREEZE_CORE;
+}
+
+uint32_t lrd_linear_bwd_plan(lrd_freeze_t f) {
+    if (f != LRD_FREEZE_NONE && f != LRD_FREEZE_U && f != LRD_FREEZE_V) return 0;
+    uint32_t plan = LRD_PLAN_DZ | LRD_PLAN_DX;
+    if (f != LRD_FREEZE_U) plan |= LRD_PLAN_DU | LRD_PLAN_DB | LRD_PLAN_NEEDS_Z;
+    if (f != LRD_FREEZE_V) plan |= LRD_PLAN_DV | LRD_PLAN_NEEDS_X;
+    return plan;
+}
+
+const char* lrd_status_string(lrd_status_t s) {
+    switch (s) {
+        case LRD_OK: return "ok";
+        case LRD_ERR_INVALID_ARG: return "invalid argument";
+        case LRD_ERR_BAD_RANK: return "rank out of range";
+        case LRD_ERR_ALIGNMENT: return "pointer not aligned";
+        case LRD_ERR_WORKSPACE: return "workspace missing or too small";
+        case LRD_ERR_UNSUPPORTED: return "unsupported geometry";
+        case LRD_ERR_ARCH: return "device is not sm_100";
+        case LRD_ERR_CUDA: return "CUDA call failed";
+        case LRD_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+lrd_status_t lrd_set_path(lrd_path_t path) {
+    if (path < LRD_PATH_AUTO || path > LRD_PATH_FUSED) return LRD_ERR_INVALID_ARG;
+    g_path.store((int)path);
+    return LRD_OK;
+}
+
+lrd_status_t lrd_check_device_status(void) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return LRD_ERR_CUDA;
+    bool raised = false;
+    if (read_and_clear_device_timeout(&raised) != LRD_OK) return LRD_ERR_CUDA;
+    return raised ? LRD_ERR_TIMEOUT : LRD_OK;
+}
+
+size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t freeze, int is_bwd) {
+    Linear L;
+    if (parse_linear(desc, &L, false) != LRD_OK) return 0;
+    (void)freeze;
+    return is_bwd ? linear_z_bytes(L) + linear_split_bytes(L) : linear_z_bytes(L);
+}
+
+size_t lrd_dense_workspace_bytes(const lrd_linear_desc_t* desc, int is_bwd) {
+    Linear L;
+    if (parse_linear(desc, &L, true) != LRD_OK) return 0;
+    if (!is_bwd || L.dt != LRD_BF16 || L.M < 1) return 256;
+    return 256 + tc_split_workspace_bytes(L.N, L.K, L.M);
+}
+
+lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
+                            const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+    Linear L;
+    LRD_TRY(parse_linear(desc, &L, false));
+    if (freeze != LRD_FREEZE_NONE && freeze != LRD_FREEZE_U && freeze != LRD_FREEZE_V) return LRD_ERR_INVALID_ARG;
+    if (!X || !V || !U || !Y) return LRD_ERR_INVALID_ARG;
+    if ((freeze == LRD_FREEZE_U) != (Z_save == nullptr)) return LRD_ERR_INVALID_ARG;
+    const void* ptrs[] = {X, V, U, bias, Y, Z_save};
+    for (const void* p : ptrs)
+        if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
+    LRD_TRY(check_ws(workspace, workspace_bytes, lrd_linear_workspace_bytes(desc, freeze, 0)));
+    LRD_TRY(check_arch());
+    if (L.M == 0) return LRD_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+
+    const int path = g_path.load();
+    if (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) {
+        ChainArgs c;
+        c.M = L.M; c.K1 = L.K; c.r = L.r; c.N2 = L.N;
+        c.In = X; c.ld_in = L.ldx; c.P = V; c.ldp = L.ldv; c.Q = U; c.ldq = L.ldu; c.bias = bias;
+        c.Out = Y; c.ld_out = L.ldy; c.T_save = Z_save; c.ldt = L.ldz; c.dtype = L.dt;
+        if (chain_eligible(c)) return chain_launch(c, s);
+    }
+    void* Z = Z_save ? Z_save : workspace;
+    const int64_t ldz = Z_save ? L.ldz : L.r;
+    LRD_TRY(run_gemm(gemm(L.M, L.r, L.K, X, L.ldx, false, V, L.ldv, true, Z, ldz, nullptr, L.dt), false, nullptr, 0, s));
+    return run_gemm(gemm(L.M, L.N, L.r, Z, ldz, false, U, L.ldu, false, Y, L.ldy, bias, L.dt), false, nullptr, 0, s);
+}
+
+lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                            const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                            lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Linear L;
+    LRD_TRY(parse_linear(desc, &L, false));
+    const uint32_t plan = lrd_linear_bwd_plan(freeze);
+    if (!plan) return LRD_ERR_INVALID_ARG;
+    if (!dY || !V || !U) return LRD_ERR_INVALID_ARG;
+    if ((plan & LRD_PLAN_NEEDS_Z) && (!Z_save || !dU)) return LRD_ERR_INVALID_ARG;
+    if ((plan & LRD_PLAN_NEEDS_X) && (!X || !dV)) return LRD_ERR_INVALID_ARG;
+    const void* ptrs[] = {dY, X, V, U, Z_save, dX, dU, dV, dbias};
+    for (const void* p : ptrs)
+        if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
+    LRD_TRY(check_ws(workspace, workspace_bytes, lrd_linear_workspace_bytes(desc, freeze, 1)));
+    LRD_TRY(check_arch());
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+
+    // frozen factor: no product is launched; a gradient buffer the caller passed reads as zero
+    if (!(plan & LRD_PLAN_DU)) {
+        LRD_TRY(zero_fill(dU, L.N, L.r, L.ldu, L.dt, s));
+        LRD_TRY(zero_fill(dbias, 1, L.N, L.N, L.dt, s));
+    }
+    if (!(plan & LRD_PLAN_DV)) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
+    if (L.M == 0) {                      // no tokens: the unfrozen gradients are sums over nothing
+        if (plan & LRD_PLAN_DU) { LRD_TRY(zero_fill(dU, L.N, L.r, L.ldu, L.dt, s)); LRD_TRY(zero_fill(dbias, 1, L.N, L.N, L.dt, s)); }
+        if (plan & LRD_PLAN_DV) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
+        return LRD_OK;
+    }
+
+    void* dZ = workspace;
+    float* partials = (float*)((uint8_t*)workspace + linear_z_bytes(L));
+    const size_t partial_bytes = workspace_bytes - linear_z_bytes(L);
+    const bool need_dz_in_memory = (plan & LRD_PLAN_DV) != 0;
+
+    bool chained = false;
+    const int path = g_path.load();
+    if (dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED)) {
+        ChainArgs c;
+        c.M = L.M; c.K1 = L.N; c.r = L.r; c.N2 = L.K;
+        c.In = dY; c.ld_in = L.ldy; c.P = U; c.ldp = L.ldu; c.Q = V; c.ldq = L.ldv; c.bias = nullptr;
+        c.Out = dX; c.ld_out = L.ldx; c.T_save = need_dz_in_memory ? dZ : nullptr; c.ldt = L.r; c.dtype = L.dt;
+        if (chain_eligible(c)) {
+            LRD_TRY(chain_launch(c, s));
+            chained = true;
+        }
+    }
+    if (!chained) {
+        if (dX || need_dz_in_memory)
+            LRD_TRY(run_gemm(gemm(L.M, L.r, L.N, dY, L.ldy, false, U, L.ldu, true, dZ, L.r, nullptr, L.dt), false, nullptr, 0, s));
+        if (dX)
+            LRD_TRY(run_gemm(gemm(L.M, L.K, L.r, dZ, L.r, false, V, L.ldv, false, dX, L.ldx, nullptr, L.dt), false, nullptr, 0, s));
+    }
+    if (plan & LRD_PLAN_DU) {
+        LRD_TRY(run_gemm(gemm(L.N, L.r, L.M, dY, L.ldy, true, Z_save, L.ldz, true, dU, L.ldu, nullptr, L.dt), true, partials,
+                         partial_bytes, s));
+        if (dbias) LRD_TRY(simt_colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, s));
+    }
+    if (plan & LRD_PLAN_DV)
+        LRD_TRY(run_gemm(gemm(L.K, L.r, L.M, X, L.ldx, true, dZ, L.r, true, dV, L.ldv, nullptr, L.dt), true, partials,
+                         partial_bytes, s));
+    return LRD_OK;
+}
+
+lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const void* W, const void* bias, void* Y,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Linear L;
+    LRD_TRY(parse_linear(desc, &L, true));
+    if (!X || !W || !Y) return LRD_ERR_INVALID_ARG;
+    (void)workspace; (void)workspace_bytes;
+    LRD_TRY(check_arch());
+    return run_gemm(gemm(L.M, L.N, L.K, X, L.ldx, false, W, L.ldv, false, Y, L.ldy, bias, L.dt), false, nullptr, 0,
+                    (cudaStream_t)cuda_stream);
+}
+
+lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* W, void* dX,
+                           void* dW, void* dbias, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Linear L;
+    LRD_TRY(parse_linear(desc, &L, true));
+    if (!dY || !X || !W || !dW) return LRD_ERR_INVALID_ARG;
+    LRD_TRY(check_ws(workspace, workspace_bytes, lrd_dense_workspace_bytes(desc, 1)));
+    LRD_TRY(check_arch());
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (L.M == 0) {
+        LRD_TRY(zero_fill(dW, L.N, L.K, L.ldv, L.dt, s));
+        return zero_fill(dbias, 1, L.N, L.N, L.dt, s);
+    }
+    float* partials = (float*)((uint8_t*)workspace + 256);
+    if (dX) LRD_TRY(run_gemm(gemm(L.M, L.K, L.N, dY, L.ldy, false, W, L.ldv, true, dX, L.ldx, nullptr, L.dt), false, nullptr, 0, s));
+    LRD_TRY(run_gemm(gemm(L.N, L.K, L.M, dY, L.ldy, true, X, L.ldx, true, dW, L.ldv, nullptr, L.dt), true, partials,
+                     workspace_bytes - 256, s));
+    if (dbias) LRD_TRY(simt_colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, s));
+    return LRD_OK;
+}
+
+size_t lrd_tucker2_workspace_bytes(const lrd_tucker2_desc_t* desc, lrd_tucker_freeze_t freeze, int is_bwd) {
+    return tucker2_workspace_bytes(desc, freeze, is_bwd);
+}
+
+lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, const void* A, const void* G,
+                             const void* Bm, const void* bias, void* Y, void* Z1_save, void* Z2_save,
+                             lrd_tucker_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    LRD_TRY(tucker2_check(desc, freeze));
+    if (!X || !A || !G || !Bm || !Y) return LRD_ERR_INVALID_ARG;
+    if ((freeze == LRD_TK_FREEZE_CORE) != (Z1_save == nullptr)) return LRD_ERR_INVALID_ARG;
+    if ((freeze == LRD_TK_FREEZE_FACTORS) != (Z2_save == nullptr)) return LRD_ERR_INVALID_ARG;
+    LRD_TRY(check_ws(workspace, workspace_bytes, tucker2_workspace_bytes(desc, freeze, 0)));
+    LRD_TRY(check_arch());
+    return tucker2_fwd(desc, X, A, G, Bm, bias, Y, Z1_save, Z2_save, freeze, workspace, workspace_bytes,
+                       g_path.load(), (cudaStream_t)cuda_stream);
+}
+
+lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, const void* X, const void* A,
+                             const void* G, const void* Bm, const void* Z1_save, const void* Z2_save, void* dX,
+                             void* dA, void* dG, void* dB, void* dbias, lrd_tucker_freeze_t freeze, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    LRD_TRY(tucker2_check(desc, freeze));
+    if (!dY || !A || !G || !Bm) return LRD_ERR_INVALID_ARG;
+    if (freeze != LRD_TK_FREEZE_FACTORS && (!X || !Z2_save || !dA || !dB)) return LRD_ERR_INVALID_ARG;
+    if (freeze != LRD_TK_FREEZE_CORE && (!Z1_save || !dG)) return LRD_ERR_INVALID_ARG;
+    LRD_TRY(check_ws(workspace, workspace_bytes, tucker2_workspace_bytes(desc, freeze, 1)));
+    LRD_TRY(check_arch());
+    return tucker2_bwd(desc, dY, X, A, G, Bm, Z1_save, Z2_save, dX, dA, dG, dB, dbias, freeze, workspace,
+                       workspace_bytes, g_path.load(), (cudaStream_t)cuda_stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,231 @@
+// General path: shared-memory tiled fp32-FMA matrix product for any shape, leading dimension and
+// operand orientation, and a deterministic column sum.  Used for fp32 layers (which must not use
+// reduced-precision tensor math) and for bf16 layers whose ranks or strides do not meet the
+// 16-byte alignment the tensor-core path needs.
+#include "common.cuh"
+#include "conv.cuh"
+
+namespace lrd {
+
+__device__ unsigned int g_device_timeout = 0;
+
+unsigned int* device_timeout_flag() {
+    static unsigned int* ptr = nullptr;
+    if (!ptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_timeout) == cudaSuccess) ptr = (unsigned int*)p;
+    }
+    return ptr;
+}
+
+lrd_status_t read_and_clear_device_timeout(bool* raised) {
+    unsigned int flag = 0;
+    if (cudaMemcpyFromSymbol(&flag, g_device_timeout, sizeof(flag)) != cudaSuccess) return LRD_ERR_CUDA;
+    *raised = flag != 0;
+    if (flag) {
+        const unsigned int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_timeout, &zero, sizeof(zero)) != cudaSuccess) return LRD_ERR_CUDA;
+    }
+    return LRD_OK;
+}
+
+namespace {
+
+constexpr int TM = 64, TN = 64, TK = 16, NT = 256;
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Operand loaders: element (m, k) of A and (k, n) of B as fp32, zero outside the problem.
+template <typename T> struct PlainA {          // [M x K] (k contiguous) or [K x M] (m contiguous)
+    const T* p; int64_t ld; int mn;
+    __device__ bool k_fastest() const { return !mn; }
+    __device__ float operator()(int64_t m, int64_t k) const { return to_f32(mn ? p[k * ld + m] : p[m * ld + k]); }
+};
+template <typename T> struct PlainB {          // [N x K] (k contiguous) or [K x N] (n contiguous)
+    const T* p; int64_t ld; int mn;
+    __device__ bool k_fastest() const { return !mn; }
+    __device__ float operator()(int64_t k, int64_t n) const { return to_f32(mn ? p[k * ld + n] : p[n * ld + k]); }
+};
+// 3x3 taps of an NHWC image as the A operand: m = pixel, k = tap * C + channel; the tap offset is
+// sign * (kh - 1, kw - 1); pixels outside the image read as zero.
+template <typename T> struct ConvTapA {
+    const T* p; int H, W, C, sign;
+    __device__ bool k_fastest() const { return true; }
+    __device__ float operator()(int64_t m, int64_t k) const {
+        const int t = (int)(k / C), c = (int)(k % C);
+        const int dh = sign * (t / 3 - 1), dw = sign * (t % 3 - 1);
+        const int w = (int)(m % W), h = (int)((m / W) % H);
+        if (h + dh < 0 || h + dh >= H || w + dw < 0 || w + dw >= W) return 0.f;
+        return to_f32(p[(m + (int64_t)dh * W + dw) * C + c]);
+    }
+};
+// One tap of an NHWC image as the B operand of the filter gradient: k = pixel, n = channel.
+template <typename T> struct ConvTapB {
+    const T* p; int H, W, C, dh, dw;
+    __device__ bool k_fastest() const { return false; }
+    __device__ float operator()(int64_t k, int64_t n) const {
+        const int w = (int)(k % W), h = (int)((k / W) % H);
+        if (h + dh < 0 || h + dh >= H || w + dw < 0 || w + dw >= W) return 0.f;
+        return to_f32(p[(k + (int64_t)dh * W + dw) * C + n]);
+    }
+};
+// The core G[o][tap][i] as the B operand of the data gradient: k = tap * Co + o, n = i.
+template <typename T> struct CoreTransposedB {
+    const T* p; int Ci, Co;
+    __device__ bool k_fastest() const { return false; }
+    __device__ float operator()(int64_t k, int64_t n) const {
+        const int64_t t = k / Co, o = k % Co;
+        return to_f32(p[(o * 9 + t) * Ci + n]);
+    }
+};
+
+template <typename T, typename LA, typename LB>
+__global__ void __launch_bounds__(NT) simt_gemm_kernel(int64_t M, int64_t N, int64_t K, const LA la, const LB lb,
+                                                       T* __restrict__ C, int64_t ldc, const T* __restrict__ bias) {
+    __shared__ float As[TK][TM + 4];
+    __shared__ float Bs[TK][TN + 4];
+    const int t = threadIdx.x;
+    const int64_t m0 = (int64_t)blockIdx.y * TM, n0 = (int64_t)blockIdx.x * TN;
+    const int tx = t % 16, ty = t / 16;  // thread computes rows ty*4.., cols tx*4..
+    float acc[4][4] = {};
+    for (int64_t k0 = 0; k0 < K; k0 += TK) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int mm, kk;
+            if (la.k_fastest()) { mm = t / 16 + 16 * i; kk = t % 16; } else { kk = t / 64 + 4 * i; mm = t % 64; }
+            const int64_t m = m0 + mm, k = k0 + kk;
+            As[kk][mm] = (m < M && k < K) ? la(m, k) : 0.f;
+            int nn;
+            if (lb.k_fastest()) { nn = t / 16 + 16 * i; kk = t % 16; } else { kk = t / 64 + 4 * i; nn = t % 64; }
+            const int64_t n = n0 + nn, kb = k0 + kk;
+            Bs[kk][nn] = (n < N && kb < K) ? lb(kb, n) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < TK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t n = n0 + tx * 4 + j;
+            if (n >= N) continue;
+            float v = acc[i][j];
+            if (bias) v += to_f32(bias[n]);
+            C[m * ldc + n] = from_f32<T>(v);
+        }
+    }
+}
+
+// out[n] = sum_m A[m][n], rows added in a fixed order (thread-strided partials, then a tree in
+// shared memory whose shape does not depend on timing).
+template <typename T>
+__global__ void __launch_bounds__(256) simt_colsum_kernel(const T* __restrict__ A, int64_t lda, int64_t M, int64_t N,
+                                                          T* __restrict__ out) {
+    __shared__ float part[8][33];
+    const int c = threadIdx.x % 32, g = threadIdx.x / 32;
+    const int64_t n = (int64_t)blockIdx.x * 32 + c;
+    float s = 0.f;
+    if (n < N)
+        for (int64_t m = g; m < M; m += 8) s += to_f32(A[m * lda + n]);
+    part[g][c] = s;
+    __syncthreads();
+    if (g == 0 && n < N) {
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += part[i][c];
+        out[n] = from_f32<T>(tot);
+    }
+}
+
+template <typename T>
+lrd_status_t simt_gemm_t(const GemmArgs& g, cudaStream_t stream) {
+    dim3 grid((unsigned)((g.N + TN - 1) / TN), (unsigned)((g.M + TM - 1) / TM));
+    PlainA<T> la{(const T*)g.A, g.lda, g.a_mn_major};
+    PlainB<T> lb{(const T*)g.B, g.ldb, g.b_mn_major};
+    simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(g.M, g.N, g.K, la, lb, (T*)g.C, g.ldc, (const T*)g.bias);
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+template <typename T>
+lrd_status_t conv_fwd_t(const void* in, const void* G, void* out, int64_t P, int H, int W, int ci, int co, int sign,
+                        bool transposed_core, cudaStream_t stream) {
+    // forward:  M = pixels, N = co, K = 9 ci, B = G as [co x 9 ci] (k contiguous)
+    // data grad: M = pixels, N = ci, K = 9 co, B = G regrouped as (tap, o) x i
+    const int64_t N = transposed_core ? ci : co, K = 9 * (int64_t)(transposed_core ? co : ci);
+    dim3 grid((unsigned)((N + TN - 1) / TN), (unsigned)((P + TM - 1) / TM));
+    ConvTapA<T> la{(const T*)in, H, W, transposed_core ? co : ci, sign};
+    if (transposed_core) {
+        CoreTransposedB<T> lb{(const T*)G, ci, co};
+        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, N, K, la, lb, (T*)out, N, (const T*)nullptr);
+    } else {
+        PlainB<T> lb{(const T*)G, 9 * (int64_t)ci, 0};
+        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, N, K, la, lb, (T*)out, N, (const T*)nullptr);
+    }
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+template <typename T>
+lrd_status_t conv_filter_t(const void* dout, const void* in, void* dG, int64_t P, int H, int W, int ci, int co,
+                           cudaStream_t stream) {
+    dim3 grid((unsigned)((ci + TN - 1) / TN), (unsigned)((co + TM - 1) / TM));
+    for (int t = 0; t < 9; ++t) {      // one product per tap: M = co, N = ci, K = pixels (single block owns all of K)
+        PlainA<T> la{(const T*)dout, co, 1};
+        ConvTapB<T> lb{(const T*)in, H, W, ci, t / 3 - 1, t % 3 - 1};
+        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(co, ci, P, la, lb, (T*)dG + (int64_t)t * ci, 9 * (int64_t)ci,
+                                                     (const T*)nullptr);
+    }
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+}  // namespace
+
+lrd_status_t simt_gemm(const GemmArgs& g, cudaStream_t stream) {
+    if (g.M <= 0 || g.N <= 0) return LRD_OK;
+    return g.dtype == LRD_F32 ? simt_gemm_t<float>(g, stream) : simt_gemm_t<__nv_bfloat16>(g, stream);
+}
+
+lrd_status_t simt_conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
+                              int64_t co, lrd_dtype_t dt, cudaStream_t s) {
+    return dt == LRD_F32 ? conv_fwd_t<float>(in, G, out, B * H * W, (int)H, (int)W, (int)ci, (int)co, 1, false, s)
+                         : conv_fwd_t<__nv_bfloat16>(in, G, out, B * H * W, (int)H, (int)W, (int)ci, (int)co, 1, false, s);
+}
+lrd_status_t simt_conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W,
+                                   int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s) {
+    return dt == LRD_F32 ? conv_fwd_t<float>(dout, G, din, B * H * W, (int)H, (int)W, (int)ci, (int)co, -1, true, s)
+                         : conv_fwd_t<__nv_bfloat16>(dout, G, din, B * H * W, (int)H, (int)W, (int)ci, (int)co, -1, true, s);
+}
+lrd_status_t simt_conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
+                                     int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s) {
+    return dt == LRD_F32 ? conv_filter_t<float>(dout, in, dG, B * H * W, (int)H, (int)W, (int)ci, (int)co, s)
+                         : conv_filter_t<__nv_bfloat16>(dout, in, dG, B * H * W, (int)H, (int)W, (int)ci, (int)co, s);
+}
+
+lrd_status_t simt_colsum(const void* A, int64_t lda, int64_t M, int64_t N, void* out, lrd_dtype_t dtype,
+                         cudaStream_t stream) {
+    if (N <= 0) return LRD_OK;
+    const unsigned grid = (unsigned)((N + 31) / 32);
+    if (dtype == LRD_F32)
+        simt_colsum_kernel<float><<<grid, 256, 0, stream>>>((const float*)A, lda, M, N, (float*)out);
+    else
+        simt_colsum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)A, lda, M, N,
+                                                                     (__nv_bfloat16*)out);
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+}  // namespace lrd

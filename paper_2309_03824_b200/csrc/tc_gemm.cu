@@ -1,0 +1,327 @@
+// Tensor-core matrix product for sm_100a: TMA -> shared memory (128-byte swizzle) ->
+// tcgen05.mma with the accumulator in tensor memory -> tcgen05.ld epilogue.
+//
+//   C[M x N] = op(A) op(B) (+ bias), bf16 in, fp32 accumulate, bf16 out; or, with a split of the
+//   reduction dimension over gridDim.z, fp32 partial tiles that a second kernel adds in a fixed
+//   order (deterministic weight gradients, no floating-point atomics).
+//
+// One 128 x BN output tile per block.  Warp 0 issues TMA loads, warp 1 owns tensor memory and
+// issues the MMAs, warps 2-5 read the accumulator (each its own quarter of the 128 lanes) and
+// store.  Both operands may be K-major (reduction index contiguous) or MN-major (row / column
+// index contiguous), which covers every product of the forward and backward pass without a
+// transposed copy.
+#include "common.cuh"
+#include "ptx.cuh"
+#include "tc.cuh"
+#include "tma.cuh"
+
+namespace lrd {
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128, BK = 64;
+constexpr int kThreads = 192;
+constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
+
+template <int BN> struct Cfg {
+    static constexpr uint32_t B_STAGE_BYTES = BN * BK * 2;
+    static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 192 ? 5 : (BN >= 128 ? 6 : 8));
+    static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack for 1024-B alignment
+    static constexpr uint32_t TMEM_COLS = BN <= 64 ? 64 : (BN <= 128 ? 128 : 256);
+};
+
+struct TcParams {
+    int64_t M, N;
+    int64_t ldp;        // leading dimension of the fp32 partial tiles (N rounded up to 4)
+    int kb_total, kb_per_split;
+    void* C;            // bf16 [M x N] (ldc) or fp32 partials [splits][M x N] packed
+    int64_t ldc;
+    const __nv_bfloat16* bias;
+    int partial;        // 1: write fp32 partials
+    unsigned int* timeout_flag;
+};
+
+template <int BN, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+    using C = Cfg<BN>;
+    constexpr int STAGES = C::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const AbortCtx ab{&abort_flag, p.timeout_flag};
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int kb_begin = blockIdx.z * p.kb_per_split;
+    const int kb_end = min(kb_begin + p.kb_per_split, p.kb_total);
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        mbar_init(smem_u32(&acc_bar), 1);
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, ab)) break;
+                const uint32_t fb = smem_u32(&full_bar[s]);
+                mbar_expect_tx(fb, C::STAGE_BYTES);
+                const uint32_t a_dst = smem_base + s * C::STAGE_BYTES;
+                const uint32_t b_dst = a_dst + A_STAGE_BYTES;
+                const int k0 = kb * BK;
+                if (A_MN) {
+#pragma unroll
+                    for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * 8192, &tmA, fb, m0 + 64 * j, k0);
+                } else {
+                    tma_load_2d(a_dst, &tmA, fb, k0, m0);
+                }
+                if (B_MN) {
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, fb, n0 + 64 * j, k0);
+                } else {
+                    tma_load_2d(b_dst, &tmB, fb, k0, n0);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(BN, A_MN, B_MN);
+            int it = 0;
+            bool ok = true;
+            for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                if (!mbar_wait(smem_u32(&full_bar[s]), ph, ab)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_src = smem_base + s * C::STAGE_BYTES;
+                const uint32_t b_src = a_src + A_STAGE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; ++kk) {
+                    const uint64_t ad = A_MN ? smem_desc_sw128(a_src + kk * 2048, 8192, 1024)
+                                             : smem_desc_sw128(a_src + kk * 32, 0, 1024);
+                    const uint64_t bd = B_MN ? smem_desc_sw128(b_src + kk * 2048, 8192, 1024)
+                                             : smem_desc_sw128(b_src + kk * 32, 0, 1024);
+                    mma_bf16_ss(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(smem_u32(&empty_bar[s]));
+            }
+            if (ok) mma_commit(smem_u32(&acc_bar));
+        }
+        __syncwarp();
+    } else {
+        const int quarter = warp % 4;                      // lanes [32 q, 32 q + 32) of tensor memory
+        const bool ready = mbar_wait(smem_u32(&acc_bar), 0, ab);
+        tc_fence_after();
+        if (ready) {
+            const int64_t row = (int64_t)m0 + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c * 32, v);
+                tmem_ld_wait();
+                const int64_t col0 = (int64_t)n0 + c * 32;
+                if (!row_ok || col0 >= p.N) continue;
+                if (p.partial) {
+                    float* dst = (float*)p.C + ((int64_t)blockIdx.z * p.M + row) * p.ldp + col0;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        if (col0 + g * 4 + 4 <= p.N) {
+                            *reinterpret_cast<uint4*>(dst + g * 4) = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                        } else {
+                            for (int e = 0; e < 4; ++e)
+                                if (col0 + g * 4 + e < p.N) dst[g * 4 + e] = __uint_as_float(v[4 * g + e]);
+                        }
+                    }
+                } else {
+                    __nv_bfloat16* dst = (__nv_bfloat16*)p.C + row * p.ldc + col0;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        float f[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            f[e] = __uint_as_float(v[8 * g + e]);
+                            if (p.bias && col0 + g * 8 + e < p.N) f[e] += __bfloat162float(p.bias[col0 + g * 8 + e]);
+                        }
+                        if (col0 + g * 8 + 8 <= p.N) {
+                            *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
+                                                                                 pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                        } else {
+                            for (int e = 0; e < 8; ++e)
+                                if (col0 + g * 8 + e < p.N) dst[g * 8 + e] = __float2bfloat16_rn(f[e]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (abort_flag) {            // give copies and MMAs still in flight time to land before freeing
+            for (int i = 0; i < 256; ++i) __nanosleep(1000);
+        }
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// out[m][n] = sum_z partial[z][m][n] (+ bias[n]), z ascending; 4 columns per thread.
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t M,
+                                                            int64_t N, int64_t ldp,
+                                                            const __nv_bfloat16* __restrict__ bias,
+                                                            __nv_bfloat16* __restrict__ C, int64_t ldc) {
+    const int64_t n4 = (N + 3) / 4;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= M * n4) return;
+    const int64_t m = idx / n4, n = (idx % n4) * 4;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const bool full = n + 4 <= N;
+    for (int z = 0; z < splits; ++z) {
+        const float* src = partial + ((int64_t)z * M + m) * ldp + n;
+        if (full) {
+            const float4 v = *reinterpret_cast<const float4*>(src);
+            acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+        } else {
+            for (int e = 0; e < 4; ++e)
+                if (n + e < N) acc[e] += src[e];
+        }
+    }
+    for (int e = 0; e < 4; ++e)
+        if (n + e < N) {
+            float v = acc[e];
+            if (bias) v += __bfloat162float(bias[n + e]);
+            C[m * ldc + n + e] = __float2bfloat16_rn(v);
+        }
+}
+
+template <int BN, bool A_MN, bool B_MN>
+lrd_status_t launch(const CUtensorMap& tA, const CUtensorMap& tB, const TcParams& p, dim3 grid, cudaStream_t stream) {
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN>;
+    static bool configured = false;     // per instantiation; the attribute is sticky per function
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_BYTES) != cudaSuccess)
+            return LRD_ERR_CUDA;
+        configured = true;
+    }
+    kern<<<grid, kThreads, Cfg<BN>::SMEM_BYTES, stream>>>(tA, tB, p);
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+template <int BN>
+lrd_status_t launch_major(bool a_mn, bool b_mn, const CUtensorMap& tA, const CUtensorMap& tB, const TcParams& p,
+                          dim3 grid, cudaStream_t s) {
+    if (a_mn) return b_mn ? launch<BN, true, true>(tA, tB, p, grid, s) : launch<BN, true, false>(tA, tB, p, grid, s);
+    return b_mn ? launch<BN, false, true>(tA, tB, p, grid, s) : launch<BN, false, false>(tA, tB, p, grid, s);
+}
+
+inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+}  // namespace
+
+bool tc_gemm_eligible(const GemmArgs& g) {
+    if (g.dtype != LRD_BF16 || g.M < 1 || g.N < 1 || g.K < 1) return false;
+    if (g.M > (int64_t)65535 * BM || g.K > (int64_t)1 << 30 || g.N > (int64_t)1 << 30) return false;
+    if (!aligned16(g.A) || !aligned16(g.B) || !aligned16(g.C)) return false;
+    if (g.lda % 8 || g.ldb % 8 || g.ldc % 8) return false;
+    return true;
+}
+
+int tc_pick_bn(int64_t M, int64_t N) {
+    const int cands[4] = {256, 192, 128, 64};
+    const int64_t mt = (M + BM - 1) / BM;
+    int best = 64;
+    double best_cost = 1e300;
+    for (int bn : cands) {
+        const int64_t tiles = mt * ((N + bn - 1) / bn);
+        const double cost = (double)((tiles + kNumSms - 1) / kNumSms) * (bn + 32);
+        if (cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+int tc_pick_splits(int64_t M, int64_t N, int64_t K) {
+    const int bn = tc_pick_bn(M, N);
+    const int64_t tiles = ((M + BM - 1) / BM) * ((N + bn - 1) / bn);
+    const int64_t kb = (K + BK - 1) / BK;
+    int64_t s = kNumSms / tiles;
+    if (s < 1) s = 1;
+    if (s > kb / 2) s = kb / 2;          // at least two k-blocks per split
+    if (s < 1) s = 1;
+    if (s > 64) s = 64;
+    // no empty split: shrink until every z has work
+    const int64_t per = (kb + s - 1) / s;
+    s = (kb + per - 1) / per;
+    return (int)s;
+}
+
+size_t tc_split_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    const int s = tc_pick_splits(M, N, K);
+    return s > 1 ? align_up((size_t)s * M * ((N + 3) / 4 * 4) * sizeof(float), 256) : 0;
+}
+
+lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes,
+                     cudaStream_t stream) {
+    if (!tc_gemm_eligible(g)) return LRD_ERR_UNSUPPORTED;
+    const int bn = tc_pick_bn(g.M, g.N);
+    int splits = allow_split ? tc_pick_splits(g.M, g.N, g.K) : 1;
+    const int64_t ldp = (g.N + 3) / 4 * 4;
+    if (splits > 1 && (!partials || partial_bytes < (size_t)splits * g.M * ldp * sizeof(float))) return LRD_ERR_WORKSPACE;
+    const int kb_total = (int)((g.K + BK - 1) / BK);
+    const int kb_per = (kb_total + splits - 1) / splits;
+
+    CUtensorMap tA, tB;
+    bool ok = g.a_mn_major ? make_tmap_2d_bf16(&tA, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, 64)
+                           : make_tmap_2d_bf16(&tA, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda, BM, BK);
+    ok = ok && (g.b_mn_major ? make_tmap_2d_bf16(&tB, g.B, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.ldb, BK, 64)
+                             : make_tmap_2d_bf16(&tB, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.ldb, (uint32_t)bn, BK));
+    if (!ok) return LRD_ERR_CUDA;
+
+    TcParams p;
+    p.M = g.M; p.N = g.N; p.ldp = ldp; p.kb_total = kb_total; p.kb_per_split = kb_per;
+    p.partial = splits > 1 ? 1 : 0;
+    p.timeout_flag = device_timeout_flag();
+    p.C = splits > 1 ? (void*)partials : g.C;
+    p.ldc = g.ldc;
+    p.bias = splits > 1 ? nullptr : (const __nv_bfloat16*)g.bias;
+    dim3 grid((unsigned)((g.N + bn - 1) / bn), (unsigned)((g.M + BM - 1) / BM), (unsigned)splits);
+    lrd_status_t st;
+    switch (bn) {
+        case 256: st = launch_major<256>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
+        case 192: st = launch_major<192>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
+        case 128: st = launch_major<128>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
+        default:  st = launch_major<64>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
+    }
+    if (st != LRD_OK || splits == 1) return st;
+    const int64_t work = g.M * ((g.N + 3) / 4);
+    splitk_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(
+        partials, splits, g.M, g.N, ldp, (const __nv_bfloat16*)g.bias, (__nv_bfloat16*)g.C, g.ldc);
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+}  // namespace lrd

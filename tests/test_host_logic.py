@@ -1,0 +1,77 @@
+"""CPU tests of the library boundary: every declared symbol is exported, and the host-only entry
+points agree bit for bit with the oracle.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from oracle import lrd_oracle as o
+from paper_2309_03824_b200 import binding as b
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "lrd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lrd_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(b.LIB_PATH)
+    names = declared_symbols()
+    assert len(names) >= 16
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(b.EXPORTS) == names
+
+
+def test_rank_quantize_bit_exact_against_oracle():
+    for m in (1, 8, 16, 32, 64, 128):
+        for r in range(1, 1300):
+            for mode in (0, 1, 2):
+                assert b.lrd_rank_quantize(r, m, mode, 1111, 2048) == o.rank_quantize(r, m, mode, 1111, 2048)
+    # error mapping
+    assert b.lrd_rank_quantize(0, 8, 0, 64, 64) == -b.LRD_ERR_INVALID_ARG
+    assert b.lrd_rank_quantize(5, 0, 0, 64, 64) == -b.LRD_ERR_INVALID_ARG
+    assert b.lrd_rank_quantize(5, 8, 9, 64, 64) == -b.LRD_ERR_INVALID_ARG
+    assert b.lrd_rank_quantize(5, 128, 0, 64, 64) == -b.LRD_ERR_BAD_RANK
+    assert b.lrd_rank_quantize(257, 64, b.LRD_ROUND_DOWN, 512, 512) == 256
+
+
+def test_freeze_schedule_and_plan_bit_exact_against_oracle():
+    for e in range(0, 50):
+        assert b.lrd_freeze_for_epoch(e) == o.freeze_for_epoch(e)
+        assert b.lrd_tucker_freeze_for_epoch(e) == o.tucker_freeze_for_epoch(e)
+    for f in (0, 1, 2):
+        assert b.lrd_linear_bwd_plan(f) == o.linear_bwd_plan(f)
+    assert b.lrd_linear_bwd_plan(7) == 0
+    assert (b.LRD_FREEZE_NONE, b.LRD_FREEZE_U, b.LRD_FREEZE_V) == (o.FREEZE_NONE, o.FREEZE_U, o.FREEZE_V)
+    assert (b.LRD_TK_FREEZE_FACTORS, b.LRD_TK_FREEZE_CORE) == (o.TK_FREEZE_FACTORS, o.TK_FREEZE_CORE)
+
+
+def test_status_strings_and_workspace_queries():
+    for s in range(9):
+        assert b.lrd_status_string(s) and b.lrd_status_string(s) != "unknown status"
+    assert b.lrd_status_string(99) == "unknown status"
+    d = b.linear_desc(4096, 768, 768, 192, b.LRD_BF16)
+    fw, bw = b.lrd_linear_workspace_bytes(d, 0, 0), b.lrd_linear_workspace_bytes(d, 0, 1)
+    assert fw >= 4096 * 192 * 2 and bw >= fw and fw % 256 == 0 and bw % 256 == 0
+    assert b.lrd_linear_workspace_bytes(b.linear_desc(16, 8, 8, 9, b.LRD_BF16), 0, 0) == 0       # rank > min(K, N)
+    assert b.lrd_linear_workspace_bytes(b.linear_desc(16, 8, 8, 4, 7), 0, 0) == 0                 # bad dtype
+    t = b.tucker2_desc(64, 14, 14, 256, 256, 96, 96, b.LRD_BF16)
+    assert b.lrd_tucker2_workspace_bytes(t, 0, 1) >= b.lrd_tucker2_workspace_bytes(t, 0, 0) > 0
+    assert b.lrd_tucker2_workspace_bytes(b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, b.LRD_F32, k=5), 0, 0) == 0
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    # NULL pointers and inconsistent masks are rejected on the host; no device is touched.
+    d = b.linear_desc(8, 16, 16, 4, b.LRD_F32)
+    assert b._lib.lrd_linear_fwd(ctypes.byref(d), None, None, None, None, None, None, 0, None, 0, None) == b.LRD_ERR_INVALID_ARG
+    bad = b.linear_desc(8, 16, 16, 17, b.LRD_F32)
+    assert b._lib.lrd_linear_fwd(ctypes.byref(bad), None, None, None, None, None, None, 0, None, 0, None) == b.LRD_ERR_BAD_RANK
+    assert b._lib.lrd_linear_bwd(ctypes.byref(d), None, None, None, None, None, None, None, None, None, 5, None, 0, None) == b.LRD_ERR_INVALID_ARG
+    with pytest.raises(b.LrdError):
+        b.lrd_set_path(17)
+    b.lrd_set_path(b.LRD_PATH_AUTO)

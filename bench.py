@@ -1,0 +1,470 @@
+#!/usr/bin/env python
+"""Benchmark of the decomposed-layer training step on B200.
+
+Default workload: the BERT-base-shaped block (four 768->768 layers at r=192, 768->3072 and
+3072->768 at r=384, M = 4096 tokens, bf16 with fp32 accumulation), forward + backward of every
+layer per step, sequential freezing alternating U-frozen / V-frozen every step.
+
+One JSON line on stdout (rank 0).  `value` is tokens/s with inputs resident in HBM; `e2e` is the
+same step with the activations copied from pinned host memory and the weight gradients copied
+back inside the timed region; `roofline` is the dominant kernel, timed alone with CUDA events;
+`cpu_baseline` is the fp64 CPU oracle timed on this machine's host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1024 * 1024
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---- algorithmic work of one layer (what the method must do; every tensor once) ------------------
+def layer_flops(M, K, N, r, freeze, which):
+    fwd = 2 * M * r * (K + N)
+    bwd = 2 * M * N * r + 2 * M * r * K + (0 if freeze == 1 else 2 * M * N * r) + (0 if freeze == 2 else 2 * M * K * r)
+    return {"fwd": fwd, "bwd": bwd, "both": fwd + bwd}[which]
+
+
+def layer_bytes(M, K, N, r, freeze, which, e=2):
+    fwd = e * (M * K + K * r + N * r + N + M * N + (0 if freeze == 1 else M * r))
+    bwd = e * (M * N + N * r + K * r + M * K)
+    if freeze != 1:
+        bwd += e * (M * r + N * r + N)
+    if freeze != 2:
+        bwd += e * (M * K + K * r)
+    return {"fwd": fwd, "bwd": bwd, "both": fwd + bwd}[which]
+
+
+# ---- clocks -----------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self, t0, t1):
+        sm, mx, reasons = [], 0, set()
+        for ts, line in self.rows:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                clk, cmax = float(f[1]), float(f[2])
+            except ValueError:
+                continue
+            mx = max(mx, cmax)
+            if t0 - 0.05 <= ts <= t1 + 0.15:
+                sm.append(clk)
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:      # timed region shorter than the sampling period: take every sample there is
+            for ts, line in self.rows:
+                f = [x.strip() for x in line.split(",")]
+                try:
+                    sm.append(float(f[1]))
+                except Exception:
+                    pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---- the oracle, timed (CPU baseline / reference arm) ------------------------------------------------
+def oracle_block_seconds(layers_np, min_seconds, max_reps=50):
+    """Forward + backward of the whole block in the fp64 oracle, alternating masks; returns
+    (seconds per step, steps run, threads used)."""
+    from oracle import lrd_oracle as o
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        freeze = o.FREEZE_U if reps % 2 == 0 else o.FREEZE_V
+        for c in layers_np:
+            Z, _ = o.linear_fwd(c["X"], c["V"], c["U"], c["b"])
+            o.linear_bwd(c["dY"], c["X"], c["V"], c["U"], Z, freeze)
+        reps += 1
+        if (time.perf_counter() - t0 >= min_seconds and reps % 2 == 0) or reps >= max_reps:
+            break
+    return (time.perf_counter() - t0) / reps, reps, threads
+
+
+def make_layers_numpy(factorize):
+    from paper_2309_03824_b200 import workloads as wl
+    cases = []
+    for i, (name, K, N, r) in enumerate(wl.C1_BERT_LAYERS):
+        c = wl.linear_case(wl.C1_M, K, N, r, "bf16", 1000 + 10 * i, wl.W_STD_TRANSFORMER, factorize)
+        c["name"] = name
+        cases.append(c)
+    return cases
+
+
+def config_dict(extra=None):
+    from paper_2309_03824_b200 import workloads as wl
+    cfg = {"workload": "configs[1]: BERT-base-shaped decomposed block, 4x(768->768,r=192)+(768->3072,r=384)+(3072->768,r=384), "
+                       "M=4096 tokens, fwd+bwd, sequential freezing alternating U-frozen/V-frozen per step",
+           "tokens_per_step": wl.C1_M, "layers": len(wl.C1_BERT_LAYERS), "ranks_quantized_to": 64}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2309_03824_b200 import workloads as wl
+
+    def np_factors(W, r):      # input construction only (the oracle's own SVD is pinned by its tests)
+        Uf, s, Vt = np.linalg.svd(W, full_matrices=False)
+        root = np.sqrt(s[:r])
+        return Vt[:r].T * root, Uf[:, :r] * root
+
+    cases = make_layers_numpy(np_factors)
+    for c in cases:
+        for k in ("X", "V", "U", "b", "dY"):
+            c[k] = c[k].astype(np.float64)
+    for _ in range(max(args.warmup, 0)):
+        oracle_block_seconds(cases, 0.0, max_reps=2)
+    steps = max(args.steps, 2)
+    steps += steps % 2
+    t0 = time.perf_counter()
+    sec, reps, threads = oracle_block_seconds(cases, 1e9, max_reps=steps)
+    total = time.perf_counter() - t0
+    val = wl.C1_M / sec
+    line = {"impl": "reference", "metric": "LRD layer fwd+bwd tokens/s", "value": val, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": reps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict({"sample": "full block, M=4096, every layer, both masks alternating"}),
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                             "sample": f"{reps} full steps of the block at M=4096 ({total:.1f} s)"},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- our arm ---------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sets", type=int, default=4, help="distinct activation buffer sets cycled through (L2 eviction)")
+    ap.add_argument("--path", default="auto", choices=["auto", "general", "unfused", "fused"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every step instead of CUDA graphs")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2309_03824_b200 import build as lrd_build
+    lrd_build.build()
+    from paper_2309_03824_b200 import binding as b
+    from paper_2309_03824_b200 import decompose
+    from paper_2309_03824_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU path exists)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks, peak_src = load_peaks()
+    b.lrd_set_path({"auto": 0, "general": 1, "unfused": 2, "fused": 3}[args.path])
+    args.warmup = max(args.warmup, 3)
+    args.steps += args.steps % 2                    # both masks equally often
+    bf = torch.bfloat16
+
+    # ---- inputs: seeded on the host, one rounding to bf16, then resident on the device -------------
+    cases = make_layers_numpy(decompose.svd_factors)
+    S = max(1, args.sets)
+    layers = []
+    act_bytes_per_set = 0
+    for c in cases:
+        M, K, N, r = c["M"], c["K"], c["N"], c["r"]
+        L = {"name": c["name"], "M": M, "K": K, "N": N, "r": r, "desc": b.linear_desc(M, K, N, r, b.LRD_BF16)}
+        L["V"], L["U"], L["b"] = (torch.from_numpy(c[k]).to("cuda", bf) for k in ("V", "U", "b"))
+        L["hX"] = torch.from_numpy(c["X"]).to(bf).pin_memory()
+        L["hdY"] = torch.from_numpy(c["dY"]).to(bf).pin_memory()
+        L["sets"] = []
+        for s in range(S):
+            st = {"X": L["hX"].to("cuda"), "dY": L["hdY"].to("cuda"),
+                  "Y": torch.empty(M, N, dtype=bf, device="cuda"), "Z": torch.empty(M, r, dtype=bf, device="cuda"),
+                  "dX": torch.empty(M, K, dtype=bf, device="cuda")}
+            L["sets"].append(st)
+        act_bytes_per_set += 2 * 2 * (M * K + M * N) + 2 * M * r
+        L["dU"] = torch.empty(N, r, dtype=bf, device="cuda")
+        L["dV"] = torch.empty(K, r, dtype=bf, device="cuda")
+        L["db"] = torch.empty(N, dtype=bf, device="cuda")
+        L["hdU"] = torch.empty(N, r, dtype=bf).pin_memory()
+        L["hdV"] = torch.empty(K, r, dtype=bf).pin_memory()
+        L["hdb"] = torch.empty(N, dtype=bf).pin_memory()
+        nws = max(b.lrd_linear_workspace_bytes(L["desc"], 0, 0), b.lrd_linear_workspace_bytes(L["desc"], 0, 1), 256)
+        L["ws"] = torch.empty(nws, dtype=torch.uint8, device="cuda")
+        layers.append(L)
+
+    def fwd(L, st, freeze):
+        b.lrd_linear_fwd(L["desc"], st["X"], L["V"], L["U"], L["b"], st["Y"], None if freeze == b.LRD_FREEZE_U else st["Z"],
+                         freeze, L["ws"])
+
+    def bwd(L, st, freeze):
+        b.lrd_linear_bwd(L["desc"], st["dY"], None if freeze == b.LRD_FREEZE_V else st["X"], L["V"], L["U"],
+                         None if freeze == b.LRD_FREEZE_U else st["Z"], st["dX"],
+                         None if freeze == b.LRD_FREEZE_U else L["dU"], None if freeze == b.LRD_FREEZE_V else L["dV"],
+                         None if freeze == b.LRD_FREEZE_U else L["db"], freeze, L["ws"])
+
+    def step_eager(s, freeze):
+        for L in layers:
+            fwd(L, L["sets"][s], freeze)
+        for L in reversed(layers):
+            bwd(L, L["sets"][s], freeze)
+
+    masks = [b.LRD_FREEZE_U, b.LRD_FREEZE_V]
+    # warm every (set, mask) once outside any capture: one-time kernel attribute set-up happens here
+    for s in range(S):
+        for f in masks:
+            step_eager(s, f)
+    torch.cuda.synchronize()
+    if b.lrd_check_device_status() != b.LRD_OK:
+        raise SystemExit("device-side wait timed out during warm-up")
+    n0 = b.lrd_launch_count()
+    step_eager(0, masks[0])
+    step_eager(0, masks[1])
+    launches_per_two_steps = b.lrd_launch_count() - n0
+
+    graphs = {}
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        for s in range(S):
+            for f in masks:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(g, stream=side):
+                        step_eager(s, f)
+                graphs[(s, f)] = g
+        torch.cuda.synchronize()
+
+    def step(i):
+        s, f = (i // 2) % S, masks[i % 2]
+        if graphs:
+            graphs[(s, f)].replay()
+        else:
+            step_eager(s, f)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        t1 = time.time()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        barrier()
+        return ms, t0, t1
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    for i in range(args.warmup):
+        step(i)
+    ms, t0, t1 = timed(step, args.steps)
+    clocks = sampler.summary(t0, t1) if rank == 0 else None
+    ms_per_step = ms / args.steps
+    tokens = wl.C1_M * world
+    value = tokens / (ms_per_step * 1e-3)
+
+    # ---- end to end: activations from pinned host memory in, weight gradients out, every step ------
+    h2d = sum(L["hX"].numel() * 2 + L["hdY"].numel() * 2 for L in layers)
+
+    def d2h_bytes(f):
+        return sum(((L["N"] * L["r"] + L["N"]) if f != b.LRD_FREEZE_U else 0) * 2 + ((L["K"] * L["r"]) if f != b.LRD_FREEZE_V else 0) * 2
+                   for L in layers)
+
+    def e2e_step(i):
+        s, f = (i // 2) % S, masks[i % 2]
+        for L in layers:
+            L["sets"][s]["X"].copy_(L["hX"], non_blocking=True)
+            L["sets"][s]["dY"].copy_(L["hdY"], non_blocking=True)
+        if graphs:
+            graphs[(s, f)].replay()
+        else:
+            step_eager(s, f)
+        for L in layers:
+            if f != b.LRD_FREEZE_U:
+                L["hdU"].copy_(L["dU"], non_blocking=True)
+                L["hdb"].copy_(L["db"], non_blocking=True)
+            if f != b.LRD_FREEZE_V:
+                L["hdV"].copy_(L["dV"], non_blocking=True)
+
+    e2e_steps = max(4, min(args.steps, 40))
+    e2e_steps += e2e_steps % 2
+    for i in range(4):
+        e2e_step(i)
+    ems, _, _ = timed(e2e_step, e2e_steps)
+    e2e_val = tokens / (ems / e2e_steps * 1e-3)
+    d2h = (d2h_bytes(masks[0]) + d2h_bytes(masks[1])) // 2
+
+    # ---- the dominant kernel alone: the fused forward chain of the widest layer (one launch per call) --
+    roof = None
+    kernels = []
+    if rank == 0:
+        reps = 40
+
+        def time_op(fn):
+            for s in range(S):
+                fn(s)
+            torch.cuda.synchronize()
+            n_before = b.lrd_launch_count()
+            fn(0)
+            n_k = b.lrd_launch_count() - n_before
+            side2 = torch.cuda.Stream()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side2):
+                with torch.cuda.graph(g, stream=side2):
+                    for s in range(S):
+                        fn(s)
+            torch.cuda.synchronize()
+            g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(reps):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e-3 / (reps * S), n_k
+
+        for L in layers[3:]:          # one attention layer and both FFN layers
+            M, K, N, r = L["M"], L["K"], L["N"], L["r"]
+            for which, f in (("fwd", b.LRD_FREEZE_U), ("bwd", b.LRD_FREEZE_U), ("bwd", b.LRD_FREEZE_V)):
+                if which == "fwd":
+                    sec, nk = time_op(lambda s, L=L, f=f: fwd(L, L["sets"][s], f))
+                else:
+                    sec, nk = time_op(lambda s, L=L, f=f: bwd(L, L["sets"][s], f))
+                fl, by = layer_flops(M, K, N, r, f, which), layer_bytes(M, K, N, r, f, which)
+                t_t, t_h = fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)
+                kernels.append({"op": f"{L['name']} {which} freeze={'U' if f == 1 else 'V'}", "kernels": nk,
+                                "us": sec * 1e6, "tflops": fl / sec / 1e12, "gbs": by / sec / 1e9,
+                                "bound": "tensor" if t_t >= t_h else "hbm", "frac": max(t_t, t_h) / sec})
+        dom = next(k for k in kernels if k["op"].startswith("ffn_1 fwd"))
+        if dom["bound"] == "tensor":
+            roof = {"bound": "tensor", "achieved": dom["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": dom["tflops"] / peaks["bf16_tflops"]}
+        else:
+            roof = {"bound": "hbm", "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": dom["gbs"] / peaks["hbm_gbs"]}
+        roof.update({"traffic": None, "kernel": dom["op"], "kernels_in_op": dom["kernels"], "peak_source": peak_src,
+                     "us_per_launch": dom["us"]})
+        for k in kernels:
+            log(json.dumps(k))
+
+    # ---- whole-step roofline (the slower of flops at the tensor peak and bytes at the HBM peak) -------
+    step_roof = {}
+    for f in masks:
+        t = 0.0
+        for L in layers:
+            for which in ("fwd", "bwd"):
+                t += max(layer_flops(L["M"], L["K"], L["N"], L["r"], f, which) / (peaks["bf16_tflops"] * 1e12),
+                         layer_bytes(L["M"], L["K"], L["N"], L["r"], f, which) / (peaks["hbm_gbs"] * 1e9))
+        step_roof[f] = t
+    t_roof = 0.5 * (step_roof[masks[0]] + step_roof[masks[1]])
+    useful_flops = 0.5 * sum(layer_flops(L["M"], L["K"], L["N"], L["r"], f, "both") for L in layers for f in masks)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        np_cases = [{k: (c[k].astype(np.float64) if isinstance(c[k], np.ndarray) else c[k]) for k in c} for c in cases]
+        sec, reps_c, threads = oracle_block_seconds(np_cases, 10.0)
+        cpu = {"value": wl.C1_M / sec, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+               "sample": f"{reps_c} full steps of the same block at M=4096, masks alternating ({sec * reps_c:.1f} s of CPU work)"}
+    if rank == 0:
+        sampler.stop()
+        line = {"metric": "LRD layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": config_dict({"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                                       "l2": f"cycling {S} activation buffer sets, {S * act_bytes_per_set / 1e6:.0f} MB > 126 MB L2",
+                                       "launch": "eager C-ABI calls" if args.no_graph else "CUDA graph replay of the C-ABI calls",
+                                       "path": args.path}),
+                "useful_tflops": useful_flops * world / (ms_per_step * 1e-3) / 1e12,
+                "step_roofline_frac": t_roof / (ms_per_step * 1e-3), "step_roofline_us": t_roof * 1e6,
+                "roofline": roof, "cpu_baseline": cpu,
+                "e2e": {"value": e2e_val, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "gpu_launches": int(launches_per_two_steps * args.steps // 2), "clocks": clocks, "peaks": peak_src}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

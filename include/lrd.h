@@ -117,6 +117,10 @@ lrd_status_t lrd_set_path(lrd_path_t path);
  * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
 lrd_status_t lrd_check_device_status(void);
 
+/* Number of kernels this library has enqueued since it was loaded (host-side counter, all
+ * streams; memset nodes of zero-filled gradients are not counted).  For launch accounting. */
+uint64_t lrd_launch_count(void);
+
 /* Scratch bytes lrd_linear_fwd (is_bwd = 0) or lrd_linear_bwd (is_bwd = 1) needs for this layer and
  * mask, for whichever path the library may take.  0 on a bad descriptor. */
 size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t freeze, int is_bwd);

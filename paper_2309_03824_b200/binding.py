@@ -27,7 +27,7 @@ LRD_PATH_AUTO, LRD_PATH_GENERAL, LRD_PATH_UNFUSED, LRD_PATH_FUSED = 0, 1, 2, 3
 
 EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
-    "lrd_status_string", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
+    "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
     "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd",
 ]
@@ -52,6 +52,8 @@ _lib.lrd_linear_bwd_plan.restype = C.c_uint32
 _lib.lrd_linear_bwd_plan.argtypes = [_int]
 _lib.lrd_status_string.restype = C.c_char_p
 _lib.lrd_status_string.argtypes = [_int]
+_lib.lrd_launch_count.restype = C.c_uint64
+_lib.lrd_launch_count.argtypes = []
 _lib.lrd_set_path.restype = _int
 _lib.lrd_set_path.argtypes = [_int]
 _lib.lrd_check_device_status.restype = _int
@@ -131,6 +133,10 @@ def lrd_linear_bwd_plan(freeze):
 
 def lrd_status_string(status):
     return _lib.lrd_status_string(int(status)).decode()
+
+
+def lrd_launch_count():
+    return int(_lib.lrd_launch_count())
 
 
 def lrd_set_path(path):

@@ -25,6 +25,9 @@ struct GemmArgs {
     lrd_dtype_t dtype;         // storage type of A, B, C, bias
 };
 
+// Host-side count of kernels enqueued (see lrd_launch_count).
+void count_launch(int n = 1);
+
 inline size_t elem_size(int dtype) { return dtype == LRD_BF16 ? 2 : 4; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

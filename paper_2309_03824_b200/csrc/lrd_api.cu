@@ -14,6 +14,7 @@ using namespace lrd;
 namespace {
 
 std::atomic<int> g_path{LRD_PATH_AUTO};
+std::atomic<uint64_t> g_launches{0};
 
 lrd_status_t check_arch() {
     int dev = 0, major = 0;
@@ -86,6 +87,8 @@ size_t linear_split_bytes(const Linear& L) {
 
 namespace lrd {
 
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n); }
+
 lrd_status_t run_gemm(const GemmArgs& g, int path, bool allow_split, float* partials, size_t partial_bytes,
                       cudaStream_t s) {
     if (g.M <= 0 || g.N <= 0) return LRD_OK;
@@ -156,6 +159,8 @@ const char* lrd_status_string(lrd_status_t s) {
     }
     return "unknown status";
 }
+
+uint64_t lrd_launch_count(void) { return g_launches.load(); }
 
 lrd_status_t lrd_set_path(lrd_path_t path) {
     if (path < LRD_PATH_AUTO || path > LRD_PATH_FUSED) return LRD_ERR_INVALID_ARG;

@@ -159,6 +159,7 @@ lrd_status_t simt_gemm_t(const GemmArgs& g, cudaStream_t stream) {
     PlainA<T> la{(const T*)g.A, g.lda, g.a_mn_major};
     PlainB<T> lb{(const T*)g.B, g.ldb, g.b_mn_major};
     simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(g.M, g.N, g.K, la, lb, (T*)g.C, g.ldc, (const T*)g.bias);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
@@ -177,6 +178,7 @@ lrd_status_t conv_fwd_t(const void* in, const void* G, void* out, int64_t P, int
         PlainB<T> lb{(const T*)G, 9 * (int64_t)ci, 0};
         simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, N, K, la, lb, (T*)out, N, (const T*)nullptr);
     }
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
@@ -190,6 +192,7 @@ lrd_status_t conv_filter_t(const void* dout, const void* in, void* dG, int64_t P
         simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(co, ci, P, la, lb, (T*)dG + (int64_t)t * ci, 9 * (int64_t)ci,
                                                      (const T*)nullptr);
     }
+    count_launch(9);
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
@@ -225,6 +228,7 @@ lrd_status_t simt_colsum(const void* A, int64_t lda, int64_t M, int64_t N, void*
     else
         simt_colsum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)A, lda, M, N,
                                                                      (__nv_bfloat16*)out);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 

@@ -230,6 +230,7 @@ lrd_status_t launch(const CUtensorMap& tA, const CUtensorMap& tB, const TcParams
         configured = true;
     }
     kern<<<grid, kThreads, Cfg<BN>::SMEM_BYTES, stream>>>(tA, tB, p);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
@@ -321,6 +322,7 @@ lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_
     const int64_t work = g.M * ((g.N + 3) / 4);
     splitk_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(
         partials, splits, g.M, g.N, ldp, (const __nv_bfloat16*)g.bias, (__nv_bfloat16*)g.C, g.ldc);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 

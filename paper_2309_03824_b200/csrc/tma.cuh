@@ -7,8 +7,9 @@
 
 namespace lrd {
 
-// 2-D bf16 tensor [rows x cols], row stride ld elements, box [box_rows x box_cols], 128-byte
-// swizzle when box_cols * 2 == 128, zero fill outside the tensor.  Returns false on failure.
+// 2-D bf16 tensor [rows x cols], row stride ld elements, box [box_rows x box_cols]; the swizzle
+// span equals the box row (128, 64 or 32 bytes; none otherwise); zero fill outside the tensor.
+// Returns false on failure.
 bool make_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld_elems,
                        uint32_t box_rows, uint32_t box_cols);
 

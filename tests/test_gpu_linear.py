@@ -41,7 +41,9 @@ def test_tensor_core_unfused_ragged_tiles(shape, freeze):
 
 
 @pytest.mark.parametrize("shape", [(300, 200, 136, 72), (128, 64, 64, 64), (513, 776, 264, 200), (640, 768, 768, 192),
-                                   (256, 3072, 768, 384), (384, 768, 3072, 384), (200, 1024, 1024, 256)])
+                                   (256, 3072, 768, 384), (384, 768, 3072, 384), (200, 1024, 1024, 256),
+                                   (5120, 256, 264, 128), (9728, 128, 136, 64), (256, 200, 136, 64), (256, 128, 128, 48),
+                                   (130, 512, 520, 512), (257, 96, 1000, 32)])
 @pytest.mark.parametrize("freeze", MASKS)
 def test_tensor_core_fused_or_auto(shape, freeze):
     M, K, N, r = shape

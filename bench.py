@@ -120,7 +120,7 @@ class ClockSampler:
 
 
 # ---- the oracle, timed (CPU baseline / reference arm) ------------------------------------------------
-def oracle_block_seconds(layers_np, min_seconds, max_reps=50):
+def oracle_block_seconds(layers_np, min_seconds, max_reps=400):
     """Forward + backward of the whole block in the fp64 oracle, alternating masks; returns
     (seconds per step, steps run, threads used)."""
     from oracle import lrd_oracle as o

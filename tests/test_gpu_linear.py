@@ -174,3 +174,32 @@ def test_dense_layer_comparison_case(shape):
     ref = o.dense_bwd(dY, X, W)
     assert rel_err(Y, o.dense_fwd(X, W, bias)) <= 2e-2
     assert rel_err(dX, ref["dX"]) <= 2e-2 and rel_err(dW, ref["dW"]) <= 2e-2 and rel_err(db, ref["db"]) <= 2e-2
+
+
+def test_fused_forward_is_one_kernel_and_keeps_z_on_chip():
+    """With U frozen the forward is a single launch (the rank-r intermediate never leaves the chip);
+    the unfused path needs two and a scratch buffer for Z."""
+    M, K, N, r = 512, 768, 768, 192
+    case = wl.random_factor_case(M, K, N, r, "bf16", 91)
+    code, tdt = DT["bf16"]
+    desc = b.linear_desc(M, K, N, r, code)
+    X, V, U, bias = (dev(case[k], "bf16") for k in ("X", "V", "U", "b"))
+    Y = torch.empty(M, N, dtype=tdt, device="cuda")
+    ws = workspace(b.lrd_linear_workspace_bytes(desc, b.LRD_FREEZE_U, 0))
+    ws.fill_(0x5A)
+    before = ws.clone()
+    b.lrd_set_path(b.LRD_PATH_FUSED)
+    try:
+        n0 = b.lrd_launch_count()
+        b.lrd_linear_fwd(desc, X, V, U, bias, Y, None, b.LRD_FREEZE_U, ws)
+        assert b.lrd_launch_count() - n0 == 1
+        torch.cuda.synchronize()
+        assert torch.equal(ws, before)                     # the workspace was not used: Z stayed on chip
+        b.lrd_set_path(b.LRD_PATH_UNFUSED)
+        n0 = b.lrd_launch_count()
+        b.lrd_linear_fwd(desc, X, V, U, bias, Y, None, b.LRD_FREEZE_U, ws)
+        assert b.lrd_launch_count() - n0 == 2
+    finally:
+        b.lrd_set_path(b.LRD_PATH_AUTO)
+    torch.cuda.synchronize()
+    assert b.lrd_check_device_status() == b.LRD_OK

@@ -1,0 +1,61 @@
+"""Run one decomposed linear layer on the GPU a few times: the smallest driver of the C ABI, for
+profilers and quick timing.
+
+    python -m paper_2309_03824_b200.run_case --M 4096 --K 768 --N 768 --r 192 --freeze U --what fwd --iters 5
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import binding as b
+from . import workloads as wl
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    for n, d in (("M", 4096), ("K", 768), ("N", 768), ("r", 192), ("iters", 5), ("sets", 8)):
+        ap.add_argument(f"--{n}", type=int, default=d)
+    ap.add_argument("--freeze", default="U", choices=["none", "U", "V"])
+    ap.add_argument("--what", default="both", choices=["fwd", "bwd", "both"])
+    ap.add_argument("--path", default="auto", choices=["auto", "general", "unfused", "fused"])
+    a = ap.parse_args()
+    freeze = {"none": 0, "U": 1, "V": 2}[a.freeze]
+    b.lrd_set_path({"auto": 0, "general": 1, "unfused": 2, "fused": 3}[a.path])
+    bf = torch.bfloat16
+    case = wl.random_factor_case(a.M, a.K, a.N, a.r, "bf16", 7)
+    V, U, bias = (torch.from_numpy(case[k]).to("cuda", bf) for k in ("V", "U", "b"))
+    desc = b.linear_desc(a.M, a.K, a.N, a.r, b.LRD_BF16)
+    ws = torch.empty(max(b.lrd_linear_workspace_bytes(desc, freeze, 1), 256), dtype=torch.uint8, device="cuda")
+    sets = []
+    for _ in range(a.sets):        # distinct buffers so that consecutive launches do not hit in L2
+        sets.append(dict(X=torch.from_numpy(case["X"]).to("cuda", bf), dY=torch.from_numpy(case["dY"]).to("cuda", bf),
+                         Y=torch.empty(a.M, a.N, dtype=bf, device="cuda"), Z=torch.empty(a.M, a.r, dtype=bf, device="cuda"),
+                         dX=torch.empty(a.M, a.K, dtype=bf, device="cuda")))
+    dU = torch.empty(a.N, a.r, dtype=bf, device="cuda")
+    dV = torch.empty(a.K, a.r, dtype=bf, device="cuda")
+    db = torch.empty(a.N, dtype=bf, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for phase in ("warm", "timed"):
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(a.iters):
+            s = sets[i % a.sets]
+            if a.what in ("fwd", "both"):
+                b.lrd_linear_fwd(desc, s["X"], V, U, bias, s["Y"], None if freeze == 1 else s["Z"], freeze, ws)
+            if a.what in ("bwd", "both"):
+                b.lrd_linear_bwd(desc, s["dY"], None if freeze == 2 else s["X"], V, U, None if freeze == 1 else s["Z"],
+                                 s["dX"], None if freeze == 1 else dU, None if freeze == 2 else dV,
+                                 None if freeze == 1 else db, freeze, ws)
+        e1.record()
+        torch.cuda.synchronize()
+    st = b.lrd_check_device_status()
+    print(f"{a.what} M={a.M} K={a.K} N={a.N} r={a.r} freeze={a.freeze} path={a.path}: "
+          f"{e0.elapsed_time(e1) * 1e3 / a.iters:.2f} us per iteration (eager launches), device status {st}")
+    if st != b.LRD_OK:
+        raise SystemExit(1)
+
+
+if __name__ == "__main__":
+    main()

@@ -10,6 +10,7 @@
 //            double-buffered in tensor memory; the epilogue adds the bias, rounds to bf16 and
 //            writes through shared memory with TMA stores (which clip the ragged edges).
 // Warp 0: TMA producer.  Warp 1: tensor memory + MMA issue.  Warps 2-5: gather and epilogue.
+// Warp 6: waits on the stage barriers for warp 1 and hands ready stages over by a named barrier.
 #include "chain.cuh"
 
 #include "ptx.cuh"
@@ -21,7 +22,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kSmemLimit = 226 * 1024;         // dynamic shared memory; the rest is left for the barriers
 constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile: 128 rows x 64 k
@@ -29,7 +30,7 @@ constexpr uint32_t kTAtomBytes = 128 * 128;         // T: 128 rows x 64 columns 
 constexpr uint32_t kStagingBytes = 4 * 2 * 4096;    // per epilogue warp: two [32 rows x 128 B] slabs
 
 struct ChainParams {
-    int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, stages, N2;
+    int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, stages, N2, G1, G2;
     uint32_t stage_bytes, t_bytes, tmem_out0, tmem_out1;
     const __nv_bfloat16* bias;
     int has_tsave;
@@ -86,87 +87,141 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int it = 0;
-            bool ok = true;
-            const int atom_cols = p.swb / 2;
-            const uint32_t p_box_bytes = 64u * p.swb;
-            for (int kb = 0; kb < p.kb1 && ok; ++kb, ++it) {
-                const int s = it % p.stages;
-                if (!mbar_wait(smem_u32(&empty_bar[s]), ((it / p.stages) & 1) ^ 1, ab)) { ok = false; break; }
-                const uint32_t fb = smem_u32(&full_bar[s]);
-                mbar_expect_tx(fb, kInTileBytes + 64u * p.RS * 2u);
-                const uint32_t dst = ring_base + s * p.stage_bytes;
-                tma_load_2d(dst, &tmIn, fb, kb * 64, m0);
-                for (int i = 0; i * atom_cols < p.RS; ++i)
-                    tma_load_2d(dst + kInTileBytes + i * p_box_bytes, &tmP, fb, c * p.RS + i * atom_cols, kb * 64);
+        // Lane 0 waits for the slot and arms its barrier; then lane l issues box l of the stage
+        // (one instruction for the warp instead of a serial chain of issues by one thread).
+        int s = 0;
+        uint32_t ph = 1;                                     // parity to wait on for an empty slot
+        bool ok = true;
+        const int atom_cols = p.swb / 2;
+        const uint32_t p_box_bytes = 64u * p.swb;
+        const int n_pbox = p.RS / atom_cols;
+        for (int kb = 0; kb < p.kb1 && ok; ++kb) {
+            const uint32_t fb = smem_u32(&full_bar[s]);
+            if (lane == 0) {
+                ok = mbar_wait(smem_u32(&empty_bar[s]), ph, ab);
+                if (ok) mbar_expect_tx(fb, kInTileBytes + 64u * p.RS * 2u);
             }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            const uint32_t dst = ring_base + s * p.stage_bytes;
+            if (lane == 0) tma_load_2d(dst, &tmIn, fb, kb * 64, m0);
+            else if (lane <= n_pbox)
+                tma_load_2d(dst + kInTileBytes + (lane - 1) * p_box_bytes, &tmP, fb, c * p.RS + (lane - 1) * atom_cols, kb * 64);
+            if (++s == p.stages) { s = 0; ph ^= 1; }
+        }
+        if (lane == 0) {
             for (int j = c; j < p.n_chunks && ok; j += p.C) {
-                for (int kb = 0; kb < p.kb2; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    if (!mbar_wait(smem_u32(&empty_bar[s]), ((it / p.stages) & 1) ^ 1, ab)) { ok = false; break; }
+                for (int kb = 0; kb < p.kb2; ++kb) {
+                    if (!mbar_wait(smem_u32(&empty_bar[s]), ph, ab)) { ok = false; break; }
                     const uint32_t fb = smem_u32(&full_bar[s]);
                     mbar_expect_tx(fb, (uint32_t)p.BN2 * 128u);
                     tma_load_2d(ring_base + s * p.stage_bytes, &tmQ, fb, kb * 64, j * p.BN2);
+                    if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int it = 0;
-            bool ok = true;
-            const uint32_t idesc1 = idesc_bf16(p.RS, false, true);
-            for (int kb = 0; kb < p.kb1; ++kb, ++it) {
-                const int s = it % p.stages;
-                if (!mbar_wait(smem_u32(&full_bar[s]), (it / p.stages) & 1, ab)) { ok = false; break; }
+        // Never waits on a barrier itself: warp 6 does the waiting and hands each group of ready
+        // stages over through a named barrier.  Both warps run the same group loops.
+        int s = 0;
+        bool ok = true;
+        const uint32_t idesc1 = idesc_bf16(p.RS, false, true);
+        for (int kb0 = 0; kb0 < p.kb1; kb0 += p.G1) {
+            const int g = min(p.G1, p.kb1 - kb0);
+            ok = !pair_sync_or(false) && ok;
+            if (lane == 0 && ok) {
                 tc_fence_after();
-                const uint32_t a_src = ring_base + s * p.stage_bytes;
-                const uint32_t b_src = a_src + kInTileBytes;
+                int ss = s;
+                for (int i = 0; i < g; ++i) {
+                    const uint32_t a_src = ring_base + ss * p.stage_bytes;
+                    const uint32_t b_src = a_src + kInTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ad = smem_desc_sw128(a_src + kk * 32, 0, 1024);
-                    const uint64_t bd = smem_desc(b_src + kk * 16 * p.swb, 64u * p.swb, 8u * p.swb, p.swb);
-                    mma_bf16_ss(tmem_base, ad, bd, idesc1, (kb > 0 || kk > 0) ? 1u : 0u);
-                }
-                mma_commit(smem_u32(&empty_bar[s]));
-            }
-            if (ok) mma_commit(smem_u32(&tacc_bar));
-            // all slices of T are in this block's shared memory once every gather warp of the cluster arrived
-            if (ok && !mbar_wait_cluster(smem_u32(&tready_bar), 0, ab)) ok = false;
-            fence_proxy_async_all();
-            tc_fence_after();
-            const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
-            int i = 0;
-            for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
-                const int buf = i & 1;
-                if (!mbar_wait(smem_u32(&out_empty[buf]), ((i >> 1) & 1) ^ 1, ab)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (buf ? p.tmem_out1 : p.tmem_out0);
-                for (int kb = 0; kb < p.kb2; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    if (!mbar_wait(smem_u32(&full_bar[s]), (it / p.stages) & 1, ab)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t b_src = ring_base + s * p.stage_bytes;
-                    const int nks = min(4, p.ks2 - kb * 4);
-                    for (int kk = 0; kk < nks; ++kk) {
-                        const uint64_t ad = smem_desc_sw128(t_base + kb * kTAtomBytes + kk * 32, 0, 1024);
-                        const uint64_t bd = smem_desc_sw128(b_src + kk * 32, 0, 1024);
-                        mma_bf16_ss(d_tmem, ad, bd, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint64_t ad = smem_desc_sw128(a_src + kk * 32, 0, 1024);
+                        const uint64_t bd = smem_desc(b_src + kk * 16 * p.swb, 64u * p.swb, 8u * p.swb, p.swb);
+                        mma_bf16_ss(tmem_base, ad, bd, idesc1, (kb0 + i > 0 || kk > 0) ? 1u : 0u);
                     }
-                    mma_commit(smem_u32(&empty_bar[s]));
+                    mma_commit(smem_u32(&empty_bar[ss]));
+                    if (++ss == p.stages) ss = 0;
                 }
-                if (ok) mma_commit(smem_u32(&out_full[buf]));
+            }
+            s = (s + g) % p.stages;
+        }
+        if (lane == 0 && ok) mma_commit(smem_u32(&tacc_bar));
+        const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
+        int i2 = 0;
+        for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
+            const int buf = i2 & 1;
+            const uint32_t d_tmem = tmem_base + (buf ? p.tmem_out1 : p.tmem_out0);
+            for (int kb0 = 0; kb0 < p.kb2; kb0 += p.G2) {
+                const int g = min(p.G2, p.kb2 - kb0);
+                // (before a chunk's first group warp 6 has also seen T complete and the accumulator buffer drained)
+                ok = !pair_sync_or(false) && ok;
+                if (lane == 0 && ok) {
+                    tc_fence_after();
+                    int ss = s;
+                    for (int i = 0; i < g; ++i) {
+                        const int kb = kb0 + i;
+                        const uint32_t b_src = ring_base + ss * p.stage_bytes;
+                        const int nks = min(4, p.ks2 - kb * 4);
+                        for (int kk = 0; kk < nks; ++kk) {
+                            const uint64_t ad = smem_desc_sw128(t_base + kb * kTAtomBytes + kk * 32, 0, 1024);
+                            const uint64_t bd = smem_desc_sw128(b_src + kk * 32, 0, 1024);
+                            mma_bf16_ss(d_tmem, ad, bd, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        mma_commit(smem_u32(&empty_bar[ss]));
+                        if (++ss == p.stages) ss = 0;
+                    }
+                    if (kb0 + g >= p.kb2) mma_commit(smem_u32(&out_full[buf]));
+                }
+                s = (s + g) % p.stages;
             }
         }
         __syncwarp();
+    } else if (warp == 6) {
+        // ------------------------------------------------------------------ waiter for the MMA issuer
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;                                      // lane 0's view; shared with warp 1 at every hand-over
+        for (int kb0 = 0; kb0 < p.kb1; kb0 += p.G1) {
+            const int g = min(p.G1, p.kb1 - kb0);
+            if (lane == 0) {
+                for (int i = 0; i < g; ++i) {
+                    if (ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
+                    if (++s == p.stages) { s = 0; ph ^= 1; }
+                }
+            }
+            __syncwarp();
+            pair_sync_or(lane == 0 && !ok);
+        }
+        int i2 = 0;
+        for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
+            const int buf = i2 & 1;
+            for (int kb0 = 0; kb0 < p.kb2; kb0 += p.G2) {
+                const int g = min(p.G2, p.kb2 - kb0);
+                if (lane == 0) {
+                    if (kb0 == 0) {
+                        // every slice of T has landed in this block's buffer; the accumulator buffer is free again
+                        if (ok && i2 == 0) ok = mbar_wait_cluster(smem_u32(&tready_bar), 0, ab);
+                        if (ok) ok = mbar_wait(smem_u32(&out_empty[buf]), ((i2 >> 1) & 1) ^ 1, ab);
+                    }
+                    for (int i = 0; i < g; ++i) {
+                        if (ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
+                        if (++s == p.stages) { s = 0; ph ^= 1; }
+                    }
+                }
+                __syncwarp();
+                pair_sync_or(lane == 0 && !ok);
+            }
+        }
     } else {
         // ------------------------------------------------------------------ gather + epilogue
         const int q = warp % 4;                              // tensor-memory lanes [32 q, 32 q + 32)
         const int row = q * 32 + lane;                       // row of the 128-row tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&tacc_bar), 0, ab));   // warp-uniform from here on
+        bool ok = mbar_wait_warp(smem_u32(&tacc_bar), 0, ab);   // warp-uniform from here on
         tc_fence_after();
         if (ok) {
             for (int piece = 0; piece * 16 < p.RS; ++piece) {
@@ -196,8 +251,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             bool got = true;
             if (lane == 0 && ok) {
                 got = mbar_wait_cluster(smem_u32(&tready_bar), 0, ab);
-                if (got) {
-                    fence_proxy_async_all();
+                if (got) {       // (the writers fenced their stores towards the async proxy before arriving)
                     for (int a = c; a < p.kb2; a += p.C) tma_store_2d(&tmT, t_base + a * kTAtomBytes, a * 64, m0);
                     tma_store_commit();
                 }
@@ -208,7 +262,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         int i = 0, sb = 0;
         for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
             const int buf = i & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&out_full[buf]), (i >> 1) & 1, ab));
+            ok = mbar_wait_warp(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = lane_addr + (buf ? p.tmem_out1 : p.tmem_out0);
@@ -222,14 +276,28 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint32_t v[32];
+                    const int colh = col0 + h * 32;
+                    // the 32 bias values of this piece: four 16-byte loads (same address in every lane),
+                    // issued before the accumulator load so that both latencies overlap
+                    uint4 bv[4] = {};
+                    const bool bias_vec = p.bias && colh + 32 <= p.N2;
+                    if (bias_vec) {
+                        const uint4* bp = reinterpret_cast<const uint4*>(p.bias + colh);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) bv[e] = __ldg(bp + e);
+                    }
                     tmem_ld_32x32(d_tmem + g * 64 + h * 32, v);
                     tmem_ld_wait();
-                    if (p.bias) {
+                    if (bias_vec) {
+                        const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const int col = col0 + h * 32 + e;
-                            if (col < p.N2) v[e] = __float_as_uint(__uint_as_float(v[e]) + __bfloat162float(p.bias[col]));
+                        for (int e = 0; e < 16; ++e) {
+                            v[2 * e] = __float_as_uint(__uint_as_float(v[2 * e]) + __uint_as_float(bw[e] << 16));
+                            v[2 * e + 1] = __float_as_uint(__uint_as_float(v[2 * e + 1]) + __uint_as_float(bw[e] & 0xFFFF0000u));
                         }
+                    } else if (p.bias) {                     // ragged last piece
+                        for (int e = 0; e < 32; ++e)
+                            if (colh + e < p.N2) v[e] = __float_as_uint(__uint_as_float(v[e]) + __bfloat162float(p.bias[colh + e]));
                     }
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc)
@@ -282,7 +350,7 @@ bool make_plan(const ChainArgs& a, Plan* out) {
     if (!aligned16(a.In) || !aligned16(a.P) || !aligned16(a.Q) || !aligned16(a.Out)) return false;
     if (a.ld_in % 8 || a.ldp % 8 || a.ldq % 8 || a.ld_out % 8) return false;
     if (a.T_save && (!aligned16(a.T_save) || a.ldt % 8)) return false;
-    if (a.bias && ((uintptr_t)a.bias & 1)) return false;
+    if (a.bias && !aligned16(a.bias)) return false;
     const int64_t tiles = (a.M + 127) / 128;
     const int t_bytes = (int)((a.r + 63) / 64) * (int)kTAtomBytes;
     Plan best{};
@@ -341,6 +409,11 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     p.ks2 = (int)a.r / 16;
     p.kb2 = (int)((a.r + 63) / 64);
     p.stages = pl.stages; p.N2 = (int)a.N2;
+    // k-blocks handed over per rendezvous: enough MMA work to cover the hand-over's own latency
+    p.G1 = pl.RS >= 176 ? 1 : 2;
+    p.G2 = pl.BN2 >= 176 ? 1 : 2;
+    if (p.G1 > pl.stages / 2) p.G1 = pl.stages / 2 > 0 ? pl.stages / 2 : 1;
+    if (p.G2 > pl.stages / 2) p.G2 = pl.stages / 2 > 0 ? pl.stages / 2 : 1;
     p.stage_bytes = pl.stage_bytes; p.t_bytes = pl.t_bytes;
     p.tmem_out0 = pl.RS <= 128 ? 128 : 256;
     p.tmem_out1 = p.tmem_out0 + (pl.RS <= 128 ? 192 : 128);

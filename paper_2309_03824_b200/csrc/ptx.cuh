@@ -50,14 +50,36 @@ struct AbortCtx {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const AbortCtx& ab) {
     for (uint32_t it = 0; it < kWaitSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it >= kWaitSpinFast) {
-            __nanosleep(128);
-            if (*ab.flag) return false;
-        }
+        __nanosleep(it < kWaitSpinFast ? 20 : 128);      // a failed try backs off: hot polling starves the issuing warps
+        if (it >= kWaitSpinFast && *ab.flag) return false;
     }
     *ab.flag = 1;
     if (ab.global_flag) atomicExch(ab.global_flag, 1u);
     return false;
+}
+
+// Warp-wide wait for the long waits of the epilogue warps: lane 0 polls with a sleep between tries
+// (hot polling by many threads competes with the producer and MMA threads for issue slots), then
+// every lane observes the completed phase itself.  Warp-uniform result.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const AbortCtx& ab) {
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) {
+        ok = false;
+        for (uint32_t it = 0; it < kWaitSpinLimit; ++it) {
+            if (mbar_try_wait(bar, parity)) { ok = true; break; }
+            __nanosleep(it < 64 ? 32 : 256);
+            if (it >= 64 && *ab.flag) break;
+        }
+        if (!ok && !*ab.flag) {
+            *ab.flag = 1;
+            if (ab.global_flag) atomicExch(ab.global_flag, 1u);
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (ok) {
+        for (int i = 0; i < 64 && !mbar_try_wait(bar, parity); ++i) {}
+    }
+    return ok;
 }
 
 // Cluster-scope variants: the arrival releases this thread's earlier writes (including writes to a
@@ -167,6 +189,18 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16])
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Rendezvous of two warps on named barrier 1 that also ORs a flag across them (no shared-memory
+// access: the MMA-issuing thread must not read shared memory between a tcgen05.commit and its
+// next MMAs, because such a read waits for the committed MMAs to finish and drains the pipe).
+// Every lane of both warps calls it, convergently.
+__device__ __forceinline__ bool pair_sync_or(bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 64, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"(flag ? 1u : 0u) : "memory");
+    return r != 0;
+}
 
 // ---- descriptors ------------------------------------------------------------------------------
 // Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.

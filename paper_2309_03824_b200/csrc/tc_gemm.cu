@@ -134,11 +134,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else {
         const int quarter = warp % 4;                      // lanes [32 q, 32 q + 32) of tensor memory
-        const bool ready = mbar_wait(smem_u32(&acc_bar), 0, ab);
+        const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
         tc_fence_after();
         if (ready) {
             const int64_t row = (int64_t)m0 + quarter * 32 + lane;
             const bool row_ok = row < p.M;
+            const bool bias_vec_ok = p.bias && (((uintptr_t)p.bias & 15u) == 0);
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
@@ -163,9 +164,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int g = 0; g < 4; ++g) {
                         float f[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            f[e] = __uint_as_float(v[8 * g + e]);
-                            if (p.bias && col0 + g * 8 + e < p.N) f[e] += __bfloat162float(p.bias[col0 + g * 8 + e]);
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * g + e]);
+                        if (p.bias) {
+                            if (bias_vec_ok && col0 + g * 8 + 8 <= p.N) {       // one 16-byte load for 8 columns
+                                const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(p.bias + col0 + g * 8));
+                                const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    f[2 * e] += __uint_as_float(bw[e] << 16);
+                                    f[2 * e + 1] += __uint_as_float(bw[e] & 0xFFFF0000u);
+                                }
+                            } else {
+                                for (int e = 0; e < 8; ++e)
+                                    if (col0 + g * 8 + e < p.N) f[e] += __bfloat162float(p.bias[col0 + g * 8 + e]);
+                            }
                         }
                         if (col0 + g * 8 + 8 <= p.N) {
                             *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),

@@ -1,0 +1,95 @@
+"""GPU parity of the Tucker-2 decomposed 3x3 convolution against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lrd_oracle as o
+from paper_2309_03824_b200 import binding as b
+from paper_2309_03824_b200 import decompose
+from paper_2309_03824_b200 import workloads as wl
+
+from helpers import DT, TOL, dev, host, rel_err, workspace
+
+pytestmark = pytest.mark.gpu
+MASKS = [b.LRD_TK_FREEZE_NONE, b.LRD_TK_FREEZE_FACTORS, b.LRD_TK_FREEZE_CORE]
+
+
+def run_tucker(case, freeze, path=b.LRD_PATH_AUTO, want_dx=True):
+    dt = case["dtype"]
+    code, tdt = DT[dt]
+    B, H, W, C, S, r1, r2 = (case[k] for k in ("B", "H", "W", "C", "S", "r1", "r2"))
+    desc = b.tucker2_desc(B, H, W, C, S, r1, r2, code)
+    X, A, G, Bm, bias, dY = (dev(case[k], dt) for k in ("X", "A", "G", "Bm", "b", "dY"))
+    ws = workspace(max(b.lrd_tucker2_workspace_bytes(desc, freeze, 0), b.lrd_tucker2_workspace_bytes(desc, freeze, 1)))
+    b.lrd_set_path(path)
+    try:
+        Y = torch.empty(B, H, W, S, dtype=tdt, device="cuda")
+        Z1 = None if freeze == b.LRD_TK_FREEZE_CORE else torch.empty(B, H, W, r1, dtype=tdt, device="cuda")
+        Z2 = None if freeze == b.LRD_TK_FREEZE_FACTORS else torch.empty(B, H, W, r2, dtype=tdt, device="cuda")
+        b.lrd_tucker2_fwd(desc, X, A, G, Bm, bias, Y, Z1, Z2, freeze, ws)
+        nan = float("nan")
+        dX = torch.full((B, H, W, C), nan, dtype=tdt, device="cuda") if want_dx else None
+        dA = torch.full((C, r1), nan, dtype=tdt, device="cuda")
+        dG = torch.full((r2, 3, 3, r1), nan, dtype=tdt, device="cuda")
+        dB = torch.full((S, r2), nan, dtype=tdt, device="cuda")
+        db = torch.full((S,), nan, dtype=tdt, device="cuda")
+        b.lrd_tucker2_bwd(desc, dY, None if freeze == b.LRD_TK_FREEZE_FACTORS else X, A, G, Bm, Z1, Z2, dX, dA, dG, dB, db,
+                          freeze, ws)
+        torch.cuda.synchronize()
+        assert b.lrd_check_device_status() == b.LRD_OK
+    finally:
+        b.lrd_set_path(b.LRD_PATH_AUTO)
+    return {"Y": Y, "Z1": Z1, "Z2": Z2, "dX": dX, "dA": dA, "dG": dG, "dB": dB, "db": db}
+
+
+def check_tucker(case, freeze, path=b.LRD_PATH_AUTO, tol=None):
+    got = run_tucker(case, freeze, path)
+    Z1, Z2, Y = o.tucker2_fwd(case["X"], case["A"], case["G"], case["Bm"], case["b"])
+    ref = o.tucker2_bwd(case["dY"], case["X"], case["A"], case["G"], case["Bm"], Z1, Z2, freeze)
+    ref.update({"Y": Y, "Z1": Z1, "Z2": Z2})
+    tol = TOL[case["dtype"]] if tol is None else tol
+    errs = {k: rel_err(v, ref[k]) for k, v in got.items() if v is not None}
+    if freeze == b.LRD_TK_FREEZE_FACTORS:
+        assert not host(got["dA"]).any() and not host(got["dB"]).any() and not host(got["db"]).any()
+    if freeze == b.LRD_TK_FREEZE_CORE:
+        assert not host(got["dG"]).any()
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, (bad, errs)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("geom", [(2, 5, 7, 12, 10, 5, 6), (1, 1, 1, 4, 4, 2, 3), (3, 14, 14, 40, 48, 24, 16)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_general_path_small_geometries(dtype, geom, freeze):
+    B, H, W, C, S, r1, r2 = geom
+    check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, dtype, 400 + H), freeze, path=b.LRD_PATH_GENERAL)
+
+
+@pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 9, 11, 128, 136, 96, 104), (5, 14, 14, 256, 256, 96, 96)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_tensor_core_path(geom, freeze):
+    B, H, W, C, S, r1, r2 = geom
+    check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 500 + C), freeze)
+
+
+@pytest.mark.parametrize("freeze", [b.LRD_TK_FREEZE_CORE, b.LRD_TK_FREEZE_FACTORS])
+def test_c3_resnet_stage3_shape_full_size(freeze):
+    c = wl.C3_TUCKER
+    case = wl.tucker_case(c["B"], c["H"], c["W"], c["C"], c["S"], c["r1"], c["r2"], c["k"], "bf16", 3000,
+                          decompose.tucker2_factors)
+    check_tucker(case, freeze)
+
+
+def test_argument_checks():
+    code, tdt = DT["bf16"]
+    d = b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, code)
+    t = torch.zeros(4096, dtype=tdt, device="cuda")
+    ws = workspace(b.lrd_tucker2_workspace_bytes(d, 0, 1))
+    # Z1_save is refused when the core is frozen and required otherwise
+    assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, t, t, b.LRD_TK_FREEZE_CORE, ws, check=False) == b.LRD_ERR_INVALID_ARG
+    assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, None, t, b.LRD_TK_FREEZE_NONE, ws, check=False) == b.LRD_ERR_INVALID_ARG
+    assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, t, t, b.LRD_TK_FREEZE_FACTORS, ws, check=False) == b.LRD_ERR_INVALID_ARG
+    bad = b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, code, k=5, pad=2)
+    assert b.lrd_tucker2_fwd(bad, t, t, t, t, None, t, t, t, 0, ws, check=False) == b.LRD_ERR_UNSUPPORTED
+    bad = b.tucker2_desc(1, 4, 4, 8, 8, 9, 4, code)
+    assert b.lrd_tucker2_fwd(bad, t, t, t, t, None, t, t, t, 0, ws, check=False) == b.LRD_ERR_BAD_RANK

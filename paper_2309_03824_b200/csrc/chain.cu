@@ -26,12 +26,12 @@ constexpr int kThreads = 224;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kSmemLimit = 226 * 1024;         // dynamic shared memory; the rest is left for the barriers
 constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile: 128 rows x 64 k
-constexpr uint32_t kTAtomBytes = 128 * 128;         // T: 128 rows x 64 columns per atom
 constexpr uint32_t kStagingBytes = 4 * 2 * 4096;    // per epilogue warp: two [32 rows x 128 B] slabs
 
 struct ChainParams {
     int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, stages, N2, G1, G2;
     uint32_t stage_bytes, t_bytes, tmem_out0, tmem_out1;
+    int taw;                  // columns per atom of the T buffer (64, 32 or 16; swizzle span = 2 * taw bytes)
     const __nv_bfloat16* bias;
     int has_tsave;
     unsigned int* timeout_flag;
@@ -52,6 +52,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     const uint32_t staging_base = t_base + p.t_bytes;
     const uint32_t ring_base = staging_base + kStagingBytes;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
+    const uint32_t t_sw = 2u * (uint32_t)p.taw, t_atom_bytes = 128u * t_sw;   // T: atoms of [128 rows x taw columns]
+    const int t_steps = p.taw / 16;                                           // MMA k-steps per atom
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int c = (int)cluster_ctarank();
     const int m0 = blockIdx.y * 128;
@@ -67,11 +69,13 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             mbar_init(smem_u32(&empty_bar[s]), 1);
         }
         mbar_init(smem_u32(&tacc_bar), 1);
-        mbar_init(smem_u32(&tready_bar), (uint32_t)p.C * 4);
+        // T complete = this block's own slice written (one arrival) + the peers' slices landed (bytes)
+        mbar_init(smem_u32(&tready_bar), 2);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&out_full[i]), 1);
             mbar_init(smem_u32(&out_empty[i]), 4);
         }
+        mbar_expect_tx(smem_u32(&tready_bar), (uint32_t)(p.C - 1) * 256u * (uint32_t)p.RS);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -167,7 +171,9 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                         const uint32_t b_src = ring_base + ss * p.stage_bytes;
                         const int nks = min(4, p.ks2 - kb * 4);
                         for (int kk = 0; kk < nks; ++kk) {
-                            const uint64_t ad = smem_desc_sw128(t_base + kb * kTAtomBytes + kk * 32, 0, 1024);
+                            const int ks = kb * 4 + kk;                       // 16-column step within T
+                            const uint64_t ad = smem_desc(t_base + (uint32_t)(ks / t_steps) * t_atom_bytes + (uint32_t)(ks % t_steps) * 32u,
+                                                          0, 8u * t_sw, t_sw);
                             const uint64_t bd = smem_desc_sw128(b_src + kk * 32, 0, 1024);
                             mma_bf16_ss(d_tmem, ad, bd, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
                         }
@@ -232,32 +238,33 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
 #pragma unroll
                 for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
                 const int gc = c * p.RS + piece * 16;        // first column of this piece within T
-                const uint32_t atom_off = (uint32_t)(gc / 64) * kTAtomBytes + (uint32_t)row * 128u;
-                const int chunk0 = (gc % 64) / 8;
-                for (int t = 0; t < p.C; ++t) {
-                    const uint32_t remote = map_to_cta(t_base + atom_off, (uint32_t)t);
+                const uint32_t row_addr = t_base + (uint32_t)(gc / p.taw) * t_atom_bytes + (uint32_t)row * t_sw;
+                const uint32_t chunk0 = (uint32_t)(gc % p.taw) / 8u;
+                const uint32_t sw_xor = (((uint32_t)row * t_sw) >> 7) & (t_sw / 16u - 1u);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        st_cluster_v4(remote + ((uint32_t)((chunk0 + h) ^ (row & 7)) << 4), w[4 * h], w[4 * h + 1],
-                                      w[4 * h + 2], w[4 * h + 3]);
-                }
+                for (int h = 0; h < 2; ++h)
+                    st_shared_v4(row_addr + (((chunk0 + h) ^ sw_xor) << 4), w[4 * h], w[4 * h + 1], w[4 * h + 2], w[4 * h + 3]);
             }
         }
-        fence_proxy_async_all();
+        // The slice [c RS, (c+1) RS) is whole atoms, i.e. one contiguous range of this block's T buffer: after
+        // the four warps have written it, one thread copies it into every peer's buffer (bulk DSMEM copy that
+        // completes on the peer's barrier) and, if asked, stores it to T_save.
+        fence_proxy_async_smem();
+        named_bar_sync(2, 128);
+        if (q == 0 && lane == 0 && ok) {
+            const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;
+            for (int t = 1; t < p.C; ++t) {
+                const uint32_t peer = (uint32_t)((c + t) % p.C);
+                dsmem_bulk_copy(slice, slice, 256u * (uint32_t)p.RS, smem_u32(&tready_bar), peer);
+            }
+            mbar_arrive(smem_u32(&tready_bar));
+            if (p.has_tsave) {
+                for (int a = 0; a * p.taw < p.RS; ++a)
+                    tma_store_2d(&tmT, slice + (uint32_t)a * t_atom_bytes, c * p.RS + a * p.taw, m0);
+                tma_store_commit();
+            }
+        }
         __syncwarp();
-        if (lane == 0 && ok)
-            for (int t = 0; t < p.C; ++t) mbar_arrive_remote(smem_u32(&tready_bar), (uint32_t)t);
-        if (p.has_tsave && q == 0) {                         // T_save: atoms a = c, c + C, ... straight from shared memory
-            bool got = true;
-            if (lane == 0 && ok) {
-                got = mbar_wait_cluster(smem_u32(&tready_bar), 0, ab);
-                if (got) {       // (the writers fenced their stores towards the async proxy before arriving)
-                    for (int a = c; a < p.kb2; a += p.C) tma_store_2d(&tmT, t_base + a * kTAtomBytes, a * 64, m0);
-                    tma_store_commit();
-                }
-            }
-            ok = __all_sync(0xffffffffu, ok && got);
-        }
         const uint32_t slab_base = staging_base + q * 8192;
         int i = 0, sb = 0;
         for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
@@ -352,7 +359,7 @@ bool make_plan(const ChainArgs& a, Plan* out) {
     if (a.T_save && (!aligned16(a.T_save) || a.ldt % 8)) return false;
     if (a.bias && !aligned16(a.bias)) return false;
     const int64_t tiles = (a.M + 127) / 128;
-    const int t_bytes = (int)((a.r + 63) / 64) * (int)kTAtomBytes;
+    const int t_bytes = (int)((a.r * 256 + 1023) / 1024 * 1024);      // 128 rows x r columns of bf16
     Plan best{};
     bool found = false;
     const int cands[3] = {4, 2, 1};
@@ -397,7 +404,7 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     ok = ok && make_tmap_2d_bf16(&tQ, a.Q, (uint64_t)a.N2, (uint64_t)a.r, (uint64_t)a.ldq, (uint32_t)pl.BN2, 64);
     ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 32, 64);
     if (a.T_save)
-        ok = ok && make_tmap_2d_bf16(&tT, a.T_save, (uint64_t)a.M, (uint64_t)a.r, (uint64_t)a.ldt, 128, 64);
+        ok = ok && make_tmap_2d_bf16(&tT, a.T_save, (uint64_t)a.M, (uint64_t)a.r, (uint64_t)a.ldt, 128, (uint32_t)pl.swb / 2);
     else
         tT = tOut;
     if (!ok) return LRD_ERR_CUDA;
@@ -415,6 +422,7 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     if (p.G1 > pl.stages / 2) p.G1 = pl.stages / 2 > 0 ? pl.stages / 2 : 1;
     if (p.G2 > pl.stages / 2) p.G2 = pl.stages / 2 > 0 ? pl.stages / 2 : 1;
     p.stage_bytes = pl.stage_bytes; p.t_bytes = pl.t_bytes;
+    p.taw = pl.swb / 2;
     p.tmem_out0 = pl.RS <= 128 ? 128 : 256;
     p.tmem_out1 = p.tmem_out0 + (pl.RS <= 128 ? 192 : 128);
     p.bias = (const __nv_bfloat16*)a.bias;

@@ -36,6 +36,12 @@ lrd_status_t simt_gemm(const GemmArgs& g, cudaStream_t stream);
 lrd_status_t simt_colsum(const void* A, int64_t lda, int64_t M, int64_t N, void* out, lrd_dtype_t dtype,
                          cudaStream_t stream);
 
+// Column sums of A[M x N] (bias gradient), rows added in a fixed order.  With `scratch` of at least
+// colsum_scratch_bytes(M, N) the sum runs in two stages over many blocks; without, in one kernel.
+size_t colsum_scratch_bytes(int64_t M, int64_t N);
+lrd_status_t colsum(const void* A, int64_t lda, int64_t M, int64_t N, void* out, lrd_dtype_t dtype, float* scratch,
+                    size_t scratch_bytes, cudaStream_t stream);
+
 // One product on the path chosen by `path` (an lrd_path_t): the tensor-core kernel when the
 // operands qualify, else the general kernel.
 lrd_status_t run_gemm(const GemmArgs& g, int path, bool allow_split, float* partials, size_t partial_bytes,

@@ -23,9 +23,14 @@ Tk parse(const lrd_tucker2_desc_t* d) {
 size_t act_bytes(const Tk& t, int64_t ch) { return align_up((size_t)(t.P > 0 ? t.P : 1) * ch * elem_size(t.dt), 256); }
 
 size_t split_bytes(const Tk& t) {
-    if (t.dt != LRD_BF16 || t.P < 1) return 0;
-    const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P), b = tc_split_workspace_bytes(t.C, t.r1, t.P);
-    return a > b ? a : b;
+    if (t.P < 1) return 0;
+    size_t need = colsum_scratch_bytes(t.P, t.S);
+    if (t.dt == LRD_BF16) {
+        const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P), b = tc_split_workspace_bytes(t.C, t.r1, t.P);
+        need = need > a ? need : a;
+        need = need > b ? need : b;
+    }
+    return need;
 }
 
 #define LRD_TRY(expr)                          \
@@ -93,7 +98,7 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
     if (factors) {
         LRD_TRY(run_gemm(make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt), path, true, partials, pbytes, s));
         LRD_TRY(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, partials, pbytes, s));
-        if (dbias) LRD_TRY(simt_colsum(dY, t.S, t.P, t.S, dbias, t.dt, s));
+        if (dbias) LRD_TRY(colsum(dY, t.S, t.P, t.S, dbias, t.dt, partials, pbytes, s));
     }
     if (core) LRD_TRY(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
     return LRD_OK;

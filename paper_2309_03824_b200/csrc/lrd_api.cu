@@ -71,10 +71,15 @@ GemmArgs gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool 
 
 size_t linear_z_bytes(const Linear& L) { return align_up((size_t)(L.M > 0 ? L.M : 1) * L.r * elem_size(L.dt), 256); }
 
-size_t linear_split_bytes(const Linear& L) {
-    if (L.dt != LRD_BF16 || L.M < 1) return 0;
-    const size_t a = tc_split_workspace_bytes(L.N, L.r, L.M), b = tc_split_workspace_bytes(L.K, L.r, L.M);
-    return a > b ? a : b;
+size_t linear_split_bytes(const Linear& L) {     // scratch after dZ: split partials of dU / dV, partial column sums
+    if (L.M < 1) return 0;
+    size_t need = colsum_scratch_bytes(L.M, L.N);
+    if (L.dt == LRD_BF16) {
+        const size_t a = tc_split_workspace_bytes(L.N, L.r, L.M), b = tc_split_workspace_bytes(L.K, L.r, L.M);
+        need = need > a ? need : a;
+        need = need > b ? need : b;
+    }
+    return need;
 }
 
 #define LRD_TRY(expr)                          \
@@ -185,8 +190,13 @@ size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t fr
 size_t lrd_dense_workspace_bytes(const lrd_linear_desc_t* desc, int is_bwd) {
     Linear L;
     if (parse_linear(desc, &L, true) != LRD_OK) return 0;
-    if (!is_bwd || L.dt != LRD_BF16 || L.M < 1) return 256;
-    return 256 + tc_split_workspace_bytes(L.N, L.K, L.M);
+    if (!is_bwd || L.M < 1) return 256;
+    size_t need = colsum_scratch_bytes(L.M, L.N);
+    if (L.dt == LRD_BF16) {
+        const size_t a = tc_split_workspace_bytes(L.N, L.K, L.M);
+        need = need > a ? need : a;
+    }
+    return 256 + need;
 }
 
 lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
@@ -274,7 +284,7 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
     if (plan & LRD_PLAN_DU) {
         LRD_TRY(run_gemm(gemm(L.N, L.r, L.M, dY, L.ldy, true, Z_save, L.ldz, true, dU, L.ldu, nullptr, L.dt), true, partials,
                          partial_bytes, s));
-        if (dbias) LRD_TRY(simt_colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, s));
+        if (dbias) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, partial_bytes, s));
     }
     if (plan & LRD_PLAN_DV)
         LRD_TRY(run_gemm(gemm(L.K, L.r, L.M, X, L.ldx, true, dZ, L.r, true, dV, L.ldv, nullptr, L.dt), true, partials,
@@ -309,7 +319,7 @@ lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const 
     if (dX) LRD_TRY(run_gemm(gemm(L.M, L.K, L.N, dY, L.ldy, false, W, L.ldv, true, dX, L.ldx, nullptr, L.dt), false, nullptr, 0, s));
     LRD_TRY(run_gemm(gemm(L.N, L.K, L.M, dY, L.ldy, true, X, L.ldx, true, dW, L.ldv, nullptr, L.dt), true, partials,
                      workspace_bytes - 256, s));
-    if (dbias) LRD_TRY(simt_colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, s));
+    if (dbias) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, workspace_bytes - 256, s));
     return LRD_OK;
 }
 

@@ -250,6 +250,20 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
+// Bulk copy from this block's shared memory into a peer block's shared memory (same offsets are the
+// caller's business); completion is counted in bytes on the peer's mbarrier.
+__device__ __forceinline__ void dsmem_bulk_copy(uint32_t dst_local_addr, uint32_t src_addr, uint32_t bytes,
+                                                uint32_t bar_local_addr, uint32_t peer_rank) {
+    asm volatile(
+        "{\n\t.reg .b32 rd, rb;\n\t"
+        "mapa.shared::cluster.u32 rd, %0, %4;\n\t"
+        "mapa.shared::cluster.u32 rb, %3, %4;\n\t"
+        "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [rd], [%1], %2, [rb];\n\t}"
+        ::"r"(dst_local_addr), "r"(src_addr), "r"(bytes), "r"(bar_local_addr), "r"(peer_rank) : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 __device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }

@@ -153,6 +153,53 @@ __global__ void __launch_bounds__(256) simt_colsum_kernel(const T* __restrict__ 
     }
 }
 
+// Two-stage column sum for tall matrices: stage 1 adds the rows of one of S row ranges for 64 columns
+// (4 row lanes per column, fixed order), stage 2 adds the S partial rows in ascending order.
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_stage1_kernel(const T* __restrict__ A, int64_t lda, int64_t M, int64_t N,
+                                                            int64_t rows_per_split, float* __restrict__ partial) {
+    __shared__ float part[4][64];
+    const int c = threadIdx.x % 64, g = threadIdx.x / 64;
+    const int64_t n = (int64_t)blockIdx.x * 64 + c;
+    const int64_t m_begin = (int64_t)blockIdx.y * rows_per_split;
+    const int64_t m_end = m_begin + rows_per_split < M ? m_begin + rows_per_split : M;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    if (n < N) {
+        int64_t m = m_begin + g;
+        for (; m + 12 < m_end; m += 16) {          // four independent loads in flight per thread
+            s0 += to_f32(A[m * lda + n]);
+            s1 += to_f32(A[(m + 4) * lda + n]);
+            s2 += to_f32(A[(m + 8) * lda + n]);
+            s3 += to_f32(A[(m + 12) * lda + n]);
+        }
+        for (; m < m_end; m += 4) s0 += to_f32(A[m * lda + n]);
+    }
+    part[g][c] = (s0 + s1) + (s2 + s3);
+    __syncthreads();
+    if (g == 0 && n < N) partial[(int64_t)blockIdx.y * N + n] = (part[0][c] + part[1][c]) + (part[2][c] + part[3][c]);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_stage2_kernel(const float* __restrict__ partial, int splits, int64_t N,
+                                                            T* __restrict__ out) {
+    const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    float tot = 0.f;
+    for (int z = 0; z < splits; ++z) tot += partial[(int64_t)z * N + n];
+    out[n] = from_f32<T>(tot);
+}
+
+template <typename T>
+lrd_status_t colsum_two_stage_t(const void* A, int64_t lda, int64_t M, int64_t N, void* out, float* scratch, int splits,
+                                cudaStream_t stream) {
+    const int64_t rows = (M + splits - 1) / splits;
+    dim3 grid((unsigned)((N + 63) / 64), (unsigned)splits);
+    colsum_stage1_kernel<T><<<grid, 256, 0, stream>>>((const T*)A, lda, M, N, rows, scratch);
+    colsum_stage2_kernel<T><<<(unsigned)((N + 255) / 256), 256, 0, stream>>>(scratch, splits, N, (T*)out);
+    count_launch(2);
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
 template <typename T>
 lrd_status_t simt_gemm_t(const GemmArgs& g, cudaStream_t stream) {
     dim3 grid((unsigned)((g.N + TN - 1) / TN), (unsigned)((g.M + TM - 1) / TM));
@@ -217,6 +264,26 @@ lrd_status_t simt_conv3x3_bwd_filter(const void* dout, const void* in, void* dG,
                                      int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s) {
     return dt == LRD_F32 ? conv_filter_t<float>(dout, in, dG, B * H * W, (int)H, (int)W, (int)ci, (int)co, s)
                          : conv_filter_t<__nv_bfloat16>(dout, in, dG, B * H * W, (int)H, (int)W, (int)ci, (int)co, s);
+}
+
+int colsum_splits(int64_t M) {
+    int64_t s = M / 64;
+    return (int)(s < 1 ? 1 : (s > 64 ? 64 : s));
+}
+
+size_t colsum_scratch_bytes(int64_t M, int64_t N) {
+    const int s = colsum_splits(M);
+    return s > 1 ? align_up((size_t)s * (size_t)N * sizeof(float), 256) : 0;
+}
+
+lrd_status_t colsum(const void* A, int64_t lda, int64_t M, int64_t N, void* out, lrd_dtype_t dtype, float* scratch,
+                    size_t scratch_bytes, cudaStream_t stream) {
+    if (N <= 0) return LRD_OK;
+    const int s = colsum_splits(M);
+    if (s > 1 && scratch && scratch_bytes >= (size_t)s * (size_t)N * sizeof(float))
+        return dtype == LRD_F32 ? colsum_two_stage_t<float>(A, lda, M, N, out, scratch, s, stream)
+                                : colsum_two_stage_t<__nv_bfloat16>(A, lda, M, N, out, scratch, s, stream);
+    return simt_colsum(A, lda, M, N, out, dtype, stream);
 }
 
 lrd_status_t simt_colsum(const void* A, int64_t lda, int64_t M, int64_t N, void* out, lrd_dtype_t dtype,

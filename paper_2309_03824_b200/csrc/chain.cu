@@ -3,14 +3,20 @@
 // A cluster of C blocks owns one 128-row tile.
 //   Phase 1  block c forms its r/C-column slice of T = In P in tensor memory (TMA-fed tcgen05.mma:
 //            In K-major, the slice of P MN-major).
-//   Gather   four warps read the slice (tcgen05.ld), round to bf16 and write it into the T buffer of
-//            every block of the cluster (distributed shared memory), in the 128-byte-swizzled
-//            K-major layout the next MMA reads.  T never goes to global memory unless T_save asks.
+//   Gather   four warps read the slice (tcgen05.ld), round it to bf16 and write it into this block's T
+//            buffer (K-major, swizzled, slices are whole atoms = one contiguous range); one thread then
+//            copies the range into every peer's T buffer with bulk DSMEM copies that complete on the
+//            peer's barrier.  T never goes to global memory unless T_save asks.
 //   Phase 2  block c forms every C-th column chunk of Out = T Q^T (T from shared memory, Q by TMA),
-//            double-buffered in tensor memory; the epilogue adds the bias, rounds to bf16 and
-//            writes through shared memory with TMA stores (which clip the ragged edges).
+//            double-buffered in tensor memory; the epilogue adds the bias, rounds to bf16 and writes
+//            through shared memory with TMA stores (which clip the ragged edges).
+// A pipeline stage holds a GROUP of 64-deep k-blocks behind one barrier pair: the cost of a stage
+// turn-around (barrier round trip, hand-over to the MMA thread, TMA issue) is per stage, not per byte,
+// so stages are made as large as shared memory allows.  The two phases lay their stages out
+// differently over the same ring.
 // Warp 0: TMA producer.  Warp 1: tensor memory + MMA issue.  Warps 2-5: gather and epilogue.
-// Warp 6: waits on the stage barriers for warp 1 and hands ready stages over by a named barrier.
+// Warp 6: waits on the stage barriers for warp 1 and hands ready stages over by a named barrier (the
+// issuing thread must not read shared memory behind a tcgen05.commit: that read waits for the MMAs).
 #include "chain.cuh"
 
 #include "ptx.cuh"
@@ -25,12 +31,14 @@ using namespace ptx;
 constexpr int kThreads = 224;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kSmemLimit = 226 * 1024;         // dynamic shared memory; the rest is left for the barriers
-constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile: 128 rows x 64 k
-constexpr uint32_t kStagingBytes = 4 * 2 * 4096;    // per epilogue warp: two [32 rows x 128 B] slabs
+constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile of one k-block: 128 rows x 64 k
+constexpr uint32_t kSlabBytes = 32 * 64;            // epilogue slab: 32 rows x 32 columns of bf16
+constexpr uint32_t kStagingBytes = 4 * 2 * kSlabBytes;
 
 struct ChainParams {
-    int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, stages, N2, G1, G2;
-    uint32_t stage_bytes, t_bytes, tmem_out0, tmem_out1;
+    int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, N2;
+    int G1, S1, G2, S2;       // k-blocks per stage and stage count of phase 1 / phase 2
+    uint32_t stage1_bytes, stage2_bytes, t_bytes;
     int taw;                  // columns per atom of the T buffer (64, 32 or 16; swizzle span = 2 * taw bytes)
     const __nv_bfloat16* bias;
     int has_tsave;
@@ -42,8 +50,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
              const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmOut,
              const __grid_constant__ CUtensorMap tmT, const ChainParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tacc_bar, tready_bar, out_full[2],
-        out_empty[2];
+    __shared__ __align__(8) uint64_t full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages],
+        tacc_bar, tready_bar, out_full[2], out_empty[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -57,6 +65,10 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int c = (int)cluster_ctarank();
     const int m0 = blockIdx.y * 128;
+    const int ng1 = (p.kb1 + p.G1 - 1) / p.G1, ng2 = (p.kb2 + p.G2 - 1) / p.G2;   // stage turns per phase / chunk
+    // phase-1 stage: G1 In tiles, then the P boxes (one per column atom, 64 G1 rows tall)
+    const uint32_t p_box_bytes = 64u * (uint32_t)p.G1 * (uint32_t)p.swb;
+    const uint32_t q_tile_bytes = (uint32_t)p.BN2 * 128u;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -64,9 +76,11 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         prefetch_tmap(&tmP);
         prefetch_tmap(&tmQ);
         prefetch_tmap(&tmOut);
-        for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), 1);
-            mbar_init(smem_u32(&empty_bar[s]), 1);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&full1[s]), 1);
+            mbar_init(smem_u32(&empty1[s]), 1);
+            mbar_init(smem_u32(&full2[s]), 1);
+            mbar_init(smem_u32(&empty2[s]), 1);
         }
         mbar_init(smem_u32(&tacc_bar), 1);
         // T complete = this block's own slice written (one arrival) + the peers' slices landed (bytes)
@@ -91,98 +105,105 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        // Lane 0 waits for the slot and arms its barrier; then lane l issues box l of the stage
-        // (one instruction for the warp instead of a serial chain of issues by one thread).
+        // Lane 0 waits for the stage and arms its barrier; then lane l issues copy l of the stage.
         int s = 0;
-        uint32_t ph = 1;                                     // parity to wait on for an empty slot
+        uint32_t ph = 1;                                     // parity to wait on for an empty stage
         bool ok = true;
         const int atom_cols = p.swb / 2;
-        const uint32_t p_box_bytes = 64u * p.swb;
         const int n_pbox = p.RS / atom_cols;
-        for (int kb = 0; kb < p.kb1 && ok; ++kb) {
-            const uint32_t fb = smem_u32(&full_bar[s]);
+        for (int g = 0; g < ng1 && ok; ++g) {
+            const uint32_t fb = smem_u32(&full1[s]);
             if (lane == 0) {
-                ok = mbar_wait(smem_u32(&empty_bar[s]), ph, ab);
-                if (ok) mbar_expect_tx(fb, kInTileBytes + 64u * p.RS * 2u);
+                ok = mbar_wait(smem_u32(&empty1[s]), ph, ab);
+                if (ok) mbar_expect_tx(fb, p.stage1_bytes);
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-            const uint32_t dst = ring_base + s * p.stage_bytes;
-            if (lane == 0) tma_load_2d(dst, &tmIn, fb, kb * 64, m0);
-            else if (lane <= n_pbox)
-                tma_load_2d(dst + kInTileBytes + (lane - 1) * p_box_bytes, &tmP, fb, c * p.RS + (lane - 1) * atom_cols, kb * 64);
-            if (++s == p.stages) { s = 0; ph ^= 1; }
+            const uint32_t dst = ring_base + s * p.stage1_bytes;
+            const int kb0 = g * p.G1;
+            if (lane < p.G1)                                 // k-blocks past K1 read as zeros
+                tma_load_2d(dst + lane * kInTileBytes, &tmIn, fb, (kb0 + lane) * 64, m0);
+            else if (lane < p.G1 + n_pbox)
+                tma_load_2d(dst + p.G1 * kInTileBytes + (lane - p.G1) * p_box_bytes, &tmP, fb,
+                            c * p.RS + (lane - p.G1) * atom_cols, kb0 * 64);
+            if (++s == p.S1) { s = 0; ph ^= 1; }
         }
-        if (lane == 0) {
-            for (int j = c; j < p.n_chunks && ok; j += p.C) {
-                for (int kb = 0; kb < p.kb2; ++kb) {
-                    if (!mbar_wait(smem_u32(&empty_bar[s]), ph, ab)) { ok = false; break; }
-                    const uint32_t fb = smem_u32(&full_bar[s]);
-                    mbar_expect_tx(fb, (uint32_t)p.BN2 * 128u);
-                    tma_load_2d(ring_base + s * p.stage_bytes, &tmQ, fb, kb * 64, j * p.BN2);
-                    if (++s == p.stages) { s = 0; ph ^= 1; }
+        // the ring is laid out anew for phase 2: wait until every phase-1 MMA has read its operands
+        if (lane == 0 && ok) ok = mbar_wait(smem_u32(&tacc_bar), 0, ab);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        s = 0;
+        ph = 1;
+        for (int j = c; j < p.n_chunks && ok; j += p.C) {
+            for (int g = 0; g < ng2; ++g) {
+                const uint32_t fb = smem_u32(&full2[s]);
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&empty2[s]), ph, ab);
+                    if (ok) mbar_expect_tx(fb, p.stage2_bytes);
                 }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                if (lane < p.G2)                             // k-blocks past r read as zeros
+                    tma_load_2d(ring_base + s * p.stage2_bytes + lane * q_tile_bytes, &tmQ, fb, (g * p.G2 + lane) * 64,
+                                j * p.BN2);
+                if (++s == p.S2) { s = 0; ph ^= 1; }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // Never waits on a barrier itself: warp 6 does the waiting and hands each group of ready
-        // stages over through a named barrier.  Both warps run the same group loops.
+        // Never waits on a barrier itself: warp 6 does the waiting and hands each ready stage over
+        // through a named barrier.  Both warps run the same loops.
         int s = 0;
         bool ok = true;
         const uint32_t idesc1 = idesc_bf16(p.RS, false, true);
-        for (int kb0 = 0; kb0 < p.kb1; kb0 += p.G1) {
-            const int g = min(p.G1, p.kb1 - kb0);
+        for (int g = 0; g < ng1; ++g) {
             ok = !pair_sync_or(false) && ok;
             if (lane == 0 && ok) {
                 tc_fence_after();
-                int ss = s;
-                for (int i = 0; i < g; ++i) {
-                    const uint32_t a_src = ring_base + ss * p.stage_bytes;
-                    const uint32_t b_src = a_src + kInTileBytes;
+                const uint32_t in_src = ring_base + s * p.stage1_bytes;
+                const uint32_t p_src = in_src + p.G1 * kInTileBytes;
+                const int nkb = min(p.G1, p.kb1 - g * p.G1);
+                for (int i = 0; i < nkb; ++i) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t ad = smem_desc_sw128(a_src + kk * 32, 0, 1024);
-                        const uint64_t bd = smem_desc(b_src + kk * 16 * p.swb, 64u * p.swb, 8u * p.swb, p.swb);
-                        mma_bf16_ss(tmem_base, ad, bd, idesc1, (kb0 + i > 0 || kk > 0) ? 1u : 0u);
+                        const uint64_t ad = smem_desc_sw128(in_src + i * kInTileBytes + kk * 32, 0, 1024);
+                        const uint64_t bd = smem_desc(p_src + (uint32_t)(i * 64 + kk * 16) * (uint32_t)p.swb, p_box_bytes,
+                                                      8u * p.swb, p.swb);
+                        mma_bf16_ss(tmem_base, ad, bd, idesc1, (g > 0 || i > 0 || kk > 0) ? 1u : 0u);
                     }
-                    mma_commit(smem_u32(&empty_bar[ss]));
-                    if (++ss == p.stages) ss = 0;
                 }
+                mma_commit(smem_u32(&empty1[s]));
             }
-            s = (s + g) % p.stages;
+            if (++s == p.S1) s = 0;
         }
         if (lane == 0 && ok) mma_commit(smem_u32(&tacc_bar));
         const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
+        s = 0;
         int i2 = 0;
         for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
-            const int buf = i2 & 1;
-            const uint32_t d_tmem = tmem_base + (buf ? p.tmem_out1 : p.tmem_out0);
-            for (int kb0 = 0; kb0 < p.kb2; kb0 += p.G2) {
-                const int g = min(p.G2, p.kb2 - kb0);
-                // (before a chunk's first group warp 6 has also seen T complete and the accumulator buffer drained)
+            const uint32_t d_tmem = tmem_base + (uint32_t)(i2 & 1) * 256u;
+            for (int g = 0; g < ng2; ++g) {
+                // (before a chunk's first stage warp 6 has also seen T complete and the accumulator buffer drained)
                 ok = !pair_sync_or(false) && ok;
                 if (lane == 0 && ok) {
                     tc_fence_after();
-                    int ss = s;
-                    for (int i = 0; i < g; ++i) {
-                        const int kb = kb0 + i;
-                        const uint32_t b_src = ring_base + ss * p.stage_bytes;
+                    const uint32_t q_src = ring_base + s * p.stage2_bytes;
+                    const int nkb = min(p.G2, p.kb2 - g * p.G2);
+                    for (int i = 0; i < nkb; ++i) {
+                        const int kb = g * p.G2 + i;
                         const int nks = min(4, p.ks2 - kb * 4);
                         for (int kk = 0; kk < nks; ++kk) {
                             const int ks = kb * 4 + kk;                       // 16-column step within T
                             const uint64_t ad = smem_desc(t_base + (uint32_t)(ks / t_steps) * t_atom_bytes + (uint32_t)(ks % t_steps) * 32u,
                                                           0, 8u * t_sw, t_sw);
-                            const uint64_t bd = smem_desc_sw128(b_src + kk * 32, 0, 1024);
+                            const uint64_t bd = smem_desc_sw128(q_src + i * q_tile_bytes + kk * 32, 0, 1024);
                             mma_bf16_ss(d_tmem, ad, bd, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
                         }
-                        mma_commit(smem_u32(&empty_bar[ss]));
-                        if (++ss == p.stages) ss = 0;
                     }
-                    if (kb0 + g >= p.kb2) mma_commit(smem_u32(&out_full[buf]));
+                    mma_commit(smem_u32(&empty2[s]));
+                    if (g == ng2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
                 }
-                s = (s + g) % p.stages;
+                if (++s == p.S2) s = 0;
             }
         }
         __syncwarp();
@@ -191,33 +212,26 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         int s = 0;
         uint32_t ph = 0;
         bool ok = true;                                      // lane 0's view; shared with warp 1 at every hand-over
-        for (int kb0 = 0; kb0 < p.kb1; kb0 += p.G1) {
-            const int g = min(p.G1, p.kb1 - kb0);
-            if (lane == 0) {
-                for (int i = 0; i < g; ++i) {
-                    if (ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
-                    if (++s == p.stages) { s = 0; ph ^= 1; }
-                }
-            }
+        for (int g = 0; g < ng1; ++g) {
+            if (lane == 0 && ok) ok = mbar_wait(smem_u32(&full1[s]), ph, ab);
+            if (++s == p.S1) { s = 0; ph ^= 1; }
             __syncwarp();
             pair_sync_or(lane == 0 && !ok);
         }
+        s = 0;
+        ph = 0;
         int i2 = 0;
         for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
-            const int buf = i2 & 1;
-            for (int kb0 = 0; kb0 < p.kb2; kb0 += p.G2) {
-                const int g = min(p.G2, p.kb2 - kb0);
+            for (int g = 0; g < ng2; ++g) {
                 if (lane == 0) {
-                    if (kb0 == 0) {
+                    if (g == 0) {
                         // every slice of T has landed in this block's buffer; the accumulator buffer is free again
                         if (ok && i2 == 0) ok = mbar_wait_cluster(smem_u32(&tready_bar), 0, ab);
-                        if (ok) ok = mbar_wait(smem_u32(&out_empty[buf]), ((i2 >> 1) & 1) ^ 1, ab);
+                        if (ok) ok = mbar_wait(smem_u32(&out_empty[i2 & 1]), ((i2 >> 1) & 1) ^ 1, ab);
                     }
-                    for (int i = 0; i < g; ++i) {
-                        if (ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
-                        if (++s == p.stages) { s = 0; ph ^= 1; }
-                    }
+                    if (ok) ok = mbar_wait(smem_u32(&full2[s]), ph, ab);
                 }
+                if (++s == p.S2) { s = 0; ph ^= 1; }
                 __syncwarp();
                 pair_sync_or(lane == 0 && !ok);
             }
@@ -248,8 +262,10 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         }
         // The slice [c RS, (c+1) RS) is whole atoms, i.e. one contiguous range of this block's T buffer: after
         // the four warps have written it, one thread copies it into every peer's buffer (bulk DSMEM copy that
-        // completes on the peer's barrier) and, if asked, stores it to T_save.
+        // completes on the peer's barrier) and, if asked, stores it to T_save.  The accumulator columns of
+        // the slice are free for phase 2 from here on.
         fence_proxy_async_smem();
+        tc_fence_before();
         named_bar_sync(2, 128);
         if (q == 0 && lane == 0 && ok) {
             const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;
@@ -265,62 +281,62 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             }
         }
         __syncwarp();
-        const uint32_t slab_base = staging_base + q * 8192;
+        // Epilogue: 32 columns at a time through a [32 rows x 64 B] slab of this warp (64-byte swizzle),
+        // two slabs in rotation; each slab leaves by its own TMA store.
+        const uint32_t slab_base = staging_base + q * 2 * kSlabBytes;
+        const uint32_t slab_row = (uint32_t)lane * 64u;
+        const uint32_t slab_xor = ((uint32_t)lane >> 1) & 3u;
         int i = 0, sb = 0;
         for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
             const int buf = i & 1;
             ok = mbar_wait_warp(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d_tmem = lane_addr + (buf ? p.tmem_out1 : p.tmem_out0);
-            for (int g = 0; g * 64 < p.BN2; ++g) {
-                const int col0 = j * p.BN2 + g * 64;
-                const uint32_t slab = slab_base + (sb & 1) * 4096;
+            const uint32_t d_tmem = lane_addr + (uint32_t)buf * 256u;
+            for (int g = 0; g * 32 < p.BN2; ++g, ++sb) {
+                const int colh = j * p.BN2 + g * 32;
+                if (colh >= p.N2) continue;                  // (uniform) nothing of this piece is inside Out
+                const uint32_t slab = slab_base + (sb & 1) * kSlabBytes;
+                // the 32 bias values of this piece: four 16-byte loads (same address in every lane), issued
+                // before the accumulator load so that both latencies overlap
+                uint4 bv[4] = {};
+                const bool bias_vec = p.bias && colh + 32 <= p.N2;
+                if (bias_vec) {
+                    const uint4* bp = reinterpret_cast<const uint4*>(p.bias + colh);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) bv[e] = __ldg(bp + e);
+                }
+                uint32_t v[32];
+                tmem_ld_32x32(d_tmem + g * 32, v);
                 if (sb >= 2) {                               // the store that last read this slab has finished reading
                     if (lane == 0) tma_store_wait_read<1>();
                     __syncwarp();
                 }
+                tmem_ld_wait();
+                if (bias_vec) {
+                    const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t v[32];
-                    const int colh = col0 + h * 32;
-                    // the 32 bias values of this piece: four 16-byte loads (same address in every lane),
-                    // issued before the accumulator load so that both latencies overlap
-                    uint4 bv[4] = {};
-                    const bool bias_vec = p.bias && colh + 32 <= p.N2;
-                    if (bias_vec) {
-                        const uint4* bp = reinterpret_cast<const uint4*>(p.bias + colh);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) bv[e] = __ldg(bp + e);
+                    for (int e = 0; e < 16; ++e) {
+                        v[2 * e] = __float_as_uint(__uint_as_float(v[2 * e]) + __uint_as_float(bw[e] << 16));
+                        v[2 * e + 1] = __float_as_uint(__uint_as_float(v[2 * e + 1]) + __uint_as_float(bw[e] & 0xFFFF0000u));
                     }
-                    tmem_ld_32x32(d_tmem + g * 64 + h * 32, v);
-                    tmem_ld_wait();
-                    if (bias_vec) {
-                        const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            v[2 * e] = __float_as_uint(__uint_as_float(v[2 * e]) + __uint_as_float(bw[e] << 16));
-                            v[2 * e + 1] = __float_as_uint(__uint_as_float(v[2 * e + 1]) + __uint_as_float(bw[e] & 0xFFFF0000u));
-                        }
-                    } else if (p.bias) {                     // ragged last piece
-                        for (int e = 0; e < 32; ++e)
-                            if (colh + e < p.N2) v[e] = __float_as_uint(__uint_as_float(v[e]) + __bfloat162float(p.bias[colh + e]));
-                    }
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc)
-                        st_shared_v4(slab + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + cc) ^ (lane & 7)) << 4),
-                                     pack_bf16(__uint_as_float(v[8 * cc]), __uint_as_float(v[8 * cc + 1])),
-                                     pack_bf16(__uint_as_float(v[8 * cc + 2]), __uint_as_float(v[8 * cc + 3])),
-                                     pack_bf16(__uint_as_float(v[8 * cc + 4]), __uint_as_float(v[8 * cc + 5])),
-                                     pack_bf16(__uint_as_float(v[8 * cc + 6]), __uint_as_float(v[8 * cc + 7])));
+                } else if (p.bias) {                         // ragged last piece
+                    for (int e = 0; e < 32; ++e)
+                        if (colh + e < p.N2) v[e] = __float_as_uint(__uint_as_float(v[e]) + __bfloat162float(p.bias[colh + e]));
                 }
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    st_shared_v4(slab + slab_row + (((uint32_t)cc ^ slab_xor) << 4),
+                                 pack_bf16(__uint_as_float(v[8 * cc]), __uint_as_float(v[8 * cc + 1])),
+                                 pack_bf16(__uint_as_float(v[8 * cc + 2]), __uint_as_float(v[8 * cc + 3])),
+                                 pack_bf16(__uint_as_float(v[8 * cc + 4]), __uint_as_float(v[8 * cc + 5])),
+                                 pack_bf16(__uint_as_float(v[8 * cc + 6]), __uint_as_float(v[8 * cc + 7])));
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0 && col0 < p.N2) {
-                    tma_store_2d(&tmOut, slab, col0, m0 + q * 32);
+                if (lane == 0) {
+                    tma_store_2d(&tmOut, slab, colh, m0 + q * 32);
                     tma_store_commit();
                 }
-                ++sb;
             }
             tc_fence_before();
             __syncwarp();
@@ -344,11 +360,25 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
 }
 
 struct Plan {
-    int C, RS, swb, BN2, stages;
-    uint32_t stage_bytes, t_bytes, smem_bytes;
+    int C, RS, swb, BN2, G1, S1, G2, S2;
+    uint32_t stage1_bytes, stage2_bytes, t_bytes, smem_bytes;
 };
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// Column chunk width of phase 2: the block with the most chunks sets the pace, so minimise
+// (chunks of the busiest block) x width; wider chunks on ties (fewer, larger copies).
+int pick_bn2(int64_t N2, int C) {
+    const int cands[3] = {256, 192, 128};
+    int best = 128;
+    int64_t best_cost = -1;
+    for (int bn : cands) {
+        const int64_t chunks = (N2 + bn - 1) / bn;
+        const int64_t cost = ((chunks + C - 1) / C) * bn;
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
 
 bool make_plan(const ChainArgs& a, Plan* out) {
     if (a.dtype != LRD_BF16 || a.M < 1 || a.K1 < 1 || a.N2 < 1) return false;
@@ -360,6 +390,7 @@ bool make_plan(const ChainArgs& a, Plan* out) {
     if (a.bias && !aligned16(a.bias)) return false;
     const int64_t tiles = (a.M + 127) / 128;
     const int t_bytes = (int)((a.r * 256 + 1023) / 1024 * 1024);      // 128 rows x r columns of bf16
+    const int kb1 = (int)((a.K1 + 63) / 64), kb2 = (int)((a.r + 63) / 64);
     Plan best{};
     bool found = false;
     const int cands[3] = {4, 2, 1};
@@ -368,16 +399,24 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         const int RS = (int)a.r / C;
         if (RS > 256) continue;
         const int swb = RS % 64 == 0 ? 128 : (RS % 32 == 0 ? 64 : 32);
-        const int BN2 = RS <= 128 ? 192 : 128;
-        uint32_t stage = kInTileBytes + 64u * RS * 2u;
-        if ((uint32_t)BN2 * 128u > stage) stage = (uint32_t)BN2 * 128u;
-        stage = (stage + 1023u) & ~1023u;
-        const int64_t room = (int64_t)kSmemLimit - 1024 - t_bytes - (int64_t)kStagingBytes;
-        int stages = (int)(room / stage);
-        if (stages > kMaxStages) stages = kMaxStages;
-        if (stages < 2) continue;
-        Plan pl{C, RS, swb, BN2, stages, stage, (uint32_t)t_bytes,
-                (uint32_t)(1024 + t_bytes + kStagingBytes + stages * stage)};
+        const int BN2 = pick_bn2(a.N2, C);
+        const int64_t ring = (int64_t)kSmemLimit - 1024 - t_bytes - (int64_t)kStagingBytes;
+        const uint32_t kb1_bytes = kInTileBytes + 128u * RS, kb2_bytes = (uint32_t)BN2 * 128u;
+        // the most k-blocks per stage that still leave two stages (phase 1: a P box is at most 256 rows)
+        int G1 = 0, G2 = 0;
+        for (int g = 4; g >= 1; --g)
+            if (ring / ((int64_t)g * kb1_bytes) >= 2) { G1 = g; break; }
+        for (int g = 4; g >= 1; --g)
+            if (ring / ((int64_t)g * kb2_bytes) >= 2) { G2 = g; break; }
+        if (!G1 || !G2) continue;
+        if (G1 > kb1) G1 = kb1;
+        if (G2 > kb2) G2 = kb2;
+        int S1 = (int)(ring / ((int64_t)G1 * kb1_bytes)), S2 = (int)(ring / ((int64_t)G2 * kb2_bytes));
+        if (S1 > kMaxStages) S1 = kMaxStages;
+        if (S2 > kMaxStages) S2 = kMaxStages;
+        const uint32_t s1b = (uint32_t)G1 * kb1_bytes, s2b = (uint32_t)G2 * kb2_bytes;
+        const uint32_t used = (uint32_t)S1 * s1b > (uint32_t)S2 * s2b ? (uint32_t)S1 * s1b : (uint32_t)S2 * s2b;
+        Plan pl{C, RS, swb, BN2, G1, S1, G2, S2, s1b, s2b, (uint32_t)t_bytes, (uint32_t)(1024 + t_bytes + kStagingBytes + used)};
         // prefer the largest cluster whose blocks are all resident at once; else the smallest feasible
         if (!found) { best = pl; found = true; }
         if (tiles * C <= kNumSms) { best = pl; break; }
@@ -400,9 +439,9 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     if (!make_plan(a, &pl)) return LRD_ERR_UNSUPPORTED;
     CUtensorMap tIn, tP, tQ, tOut, tT;
     bool ok = make_tmap_2d_bf16(&tIn, a.In, (uint64_t)a.M, (uint64_t)a.K1, (uint64_t)a.ld_in, 128, 64);
-    ok = ok && make_tmap_2d_bf16(&tP, a.P, (uint64_t)a.K1, (uint64_t)a.r, (uint64_t)a.ldp, 64, (uint32_t)pl.swb / 2);
+    ok = ok && make_tmap_2d_bf16(&tP, a.P, (uint64_t)a.K1, (uint64_t)a.r, (uint64_t)a.ldp, 64u * (uint32_t)pl.G1, (uint32_t)pl.swb / 2);
     ok = ok && make_tmap_2d_bf16(&tQ, a.Q, (uint64_t)a.N2, (uint64_t)a.r, (uint64_t)a.ldq, (uint32_t)pl.BN2, 64);
-    ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 32, 64);
+    ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 32, 32);
     if (a.T_save)
         ok = ok && make_tmap_2d_bf16(&tT, a.T_save, (uint64_t)a.M, (uint64_t)a.r, (uint64_t)a.ldt, 128, (uint32_t)pl.swb / 2);
     else
@@ -415,16 +454,10 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     p.kb1 = (int)((a.K1 + 63) / 64);
     p.ks2 = (int)a.r / 16;
     p.kb2 = (int)((a.r + 63) / 64);
-    p.stages = pl.stages; p.N2 = (int)a.N2;
-    // k-blocks handed over per rendezvous: enough MMA work to cover the hand-over's own latency
-    p.G1 = pl.RS >= 176 ? 1 : 2;
-    p.G2 = pl.BN2 >= 176 ? 1 : 2;
-    if (p.G1 > pl.stages / 2) p.G1 = pl.stages / 2 > 0 ? pl.stages / 2 : 1;
-    if (p.G2 > pl.stages / 2) p.G2 = pl.stages / 2 > 0 ? pl.stages / 2 : 1;
-    p.stage_bytes = pl.stage_bytes; p.t_bytes = pl.t_bytes;
+    p.N2 = (int)a.N2;
+    p.G1 = pl.G1; p.S1 = pl.S1; p.G2 = pl.G2; p.S2 = pl.S2;
+    p.stage1_bytes = pl.stage1_bytes; p.stage2_bytes = pl.stage2_bytes; p.t_bytes = pl.t_bytes;
     p.taw = pl.swb / 2;
-    p.tmem_out0 = pl.RS <= 128 ? 128 : 256;
-    p.tmem_out1 = p.tmem_out0 + (pl.RS <= 128 ? 192 : 128);
     p.bias = (const __nv_bfloat16*)a.bias;
     p.has_tsave = a.T_save ? 1 : 0;
     p.timeout_flag = device_timeout_flag();

@@ -7,7 +7,7 @@
 //
 // One 128 x BN output tile per block.  Warp 0 issues TMA loads, warp 1 owns tensor memory and
 // issues the MMAs, warps 2-5 read the accumulator (each its own quarter of the 128 lanes) and
-// store.  Both operands may be K-major (reduction index contiguous) or MN-major (row / column
+// store, warp 6 waits on the stage barriers for warp 1.  Both operands may be K-major (reduction index contiguous) or MN-major (row / column
 // index contiguous), which covers every product of the forward and backward pass without a
 // transposed copy.
 #include "common.cuh"
@@ -21,7 +21,7 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
 
 template <int BN> struct Cfg {
@@ -108,14 +108,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(BN, A_MN, B_MN);
-            int it = 0;
-            bool ok = true;
-            for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
-                if (!mbar_wait(smem_u32(&full_bar[s]), ph, ab)) { ok = false; break; }
+        // MMA issuer.  It never waits on a barrier itself (a shared-memory read behind a tcgen05.commit
+        // stalls until the committed MMAs finish): warp 6 waits and hands each ready stage over.
+        constexpr uint32_t idesc = idesc_bf16(BN, A_MN, B_MN);
+        int s = 0;
+        bool ok = true;
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+            ok = !pair_sync_or(false) && ok;
+            if (lane == 0 && ok) {
                 tc_fence_after();
                 const uint32_t a_src = smem_base + s * C::STAGE_BYTES;
                 const uint32_t b_src = a_src + A_STAGE_BYTES;
@@ -125,13 +125,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                              : smem_desc_sw128(a_src + kk * 32, 0, 1024);
                     const uint64_t bd = B_MN ? smem_desc_sw128(b_src + kk * 2048, 8192, 1024)
                                              : smem_desc_sw128(b_src + kk * 32, 0, 1024);
-                    mma_bf16_ss(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    mma_bf16_ss(tmem_base, ad, bd, idesc, (kb > kb_begin || kk > 0) ? 1u : 0u);
                 }
                 mma_commit(smem_u32(&empty_bar[s]));
             }
-            if (ok) mma_commit(smem_u32(&acc_bar));
+            if (++s == STAGES) s = 0;
         }
+        if (lane == 0 && ok) mma_commit(smem_u32(&acc_bar));
         __syncwarp();
+    } else if (warp == 6) {
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+            if (lane == 0 && ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
+            if (++s == STAGES) { s = 0; ph ^= 1; }
+            __syncwarp();
+            pair_sync_or(lane == 0 && !ok);
+        }
     } else {
         const int quarter = warp % 4;                      // lanes [32 q, 32 q + 32) of tensor memory
         const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
@@ -265,26 +276,34 @@ bool tc_gemm_eligible(const GemmArgs& g) {
     return true;
 }
 
-int tc_pick_bn(int64_t M, int64_t N) {
+// Tile width.  One k-block of a 128 x BN tile costs four MMAs of max(77, BN / 2) cycles each (an MMA
+// narrower than 154 columns is issue-bound), so a 64-wide tile is as slow as a 128-wide one.
+//   split = false: blocks run in waves over the SMs -> minimise waves x per-tile cost;
+//   split = true:  the reduction is split until the machine is full -> minimise tiles x per-tile cost.
+static int pick_bn(int64_t M, int64_t N, bool split) {
     const int cands[4] = {256, 192, 128, 64};
     const int64_t mt = (M + BM - 1) / BM;
     int best = 64;
     double best_cost = 1e300;
     for (int bn : cands) {
+        if (bn == 64 && N > 64) continue;
         const int64_t tiles = mt * ((N + bn - 1) / bn);
-        const double cost = (double)((tiles + kNumSms - 1) / kNumSms) * (bn + 32);
+        const double per_tile = bn < 154 ? 154.0 : (double)bn;
+        const double cost = split ? (double)tiles * per_tile : (double)((tiles + kNumSms - 1) / kNumSms) * (per_tile + 32);
         if (cost < best_cost) { best_cost = cost; best = bn; }
     }
     return best;
 }
 
+int tc_pick_bn(int64_t M, int64_t N) { return pick_bn(M, N, false); }
+
 int tc_pick_splits(int64_t M, int64_t N, int64_t K) {
-    const int bn = tc_pick_bn(M, N);
+    const int bn = pick_bn(M, N, true);
     const int64_t tiles = ((M + BM - 1) / BM) * ((N + bn - 1) / bn);
     const int64_t kb = (K + BK - 1) / BK;
     int64_t s = kNumSms / tiles;
     if (s < 1) s = 1;
-    if (s > kb / 2) s = kb / 2;          // at least two k-blocks per split
+    if (s > kb / 4) s = kb / 4;          // at least four k-blocks per split
     if (s < 1) s = 1;
     if (s > 64) s = 64;
     // no empty split: shrink until every z has work
@@ -301,8 +320,8 @@ size_t tc_split_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes,
                      cudaStream_t stream) {
     if (!tc_gemm_eligible(g)) return LRD_ERR_UNSUPPORTED;
-    const int bn = tc_pick_bn(g.M, g.N);
     int splits = allow_split ? tc_pick_splits(g.M, g.N, g.K) : 1;
+    const int bn = pick_bn(g.M, g.N, splits > 1);
     const int64_t ldp = (g.N + 3) / 4 * 4;
     if (splits > 1 && (!partials || partial_bytes < (size_t)splits * g.M * ldp * sizeof(float))) return LRD_ERR_WORKSPACE;
     const int kb_total = (int)((g.K + BK - 1) / BK);

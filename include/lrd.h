@@ -48,7 +48,8 @@ typedef enum {
     LRD_ERR_UNSUPPORTED = 5,  /* convolution geometry other than k = 3, stride 1, pad 1 */
     LRD_ERR_ARCH = 6,         /* current device is not sm_100 */
     LRD_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
-    LRD_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out (see lrd_check_device_status) */
+    LRD_ERR_TIMEOUT = 8,      /* a bounded device-side wait ran out (see lrd_check_device_status) */
+    LRD_ERR_TOO_LARGE = 9     /* a size exceeds the fixed limit of an entry point that brings its own scratch */
 } lrd_status_t;
 
 typedef enum { LRD_F32 = 0, LRD_BF16 = 1 } lrd_dtype_t;
@@ -156,6 +157,32 @@ lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const v
 /* dX = dY W (NULL skips), dW = dY^T X, dbias = column sums of dY (NULL skips). */
 lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* W, void* dX,
                            void* dW, void* dbias, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- bias gradient for callers that cannot allocate device memory --------------------------- */
+
+/* The paper has no counterpart for this entry point; it exists for the sake of its callers.
+ *
+ * dbias[N] = column sums of dY[M x N] (leading dimension ldy, 0 = packed), the same quantity and the
+ * same kernels as the dbias output of lrd_linear_bwd, but WITHOUT a workspace argument: the partial
+ * sums go to a fixed 2 MiB array that lives inside the library's device image.  It is meant for code
+ * that has no way to obtain scratch memory when it needs the result - for instance a plug-in that is
+ * handed ready-made tensors by a framework whose allocator it must not call, a callback running where
+ * cudaMalloc is forbidden, or a process whose memory pool is already fully committed.  The function
+ * itself calls no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ *  - Limit: N <= 8192 (the array holds 64 partial rows of that width); larger N returns
+ *    LRD_ERR_TOO_LARGE and nothing is launched.  M is unlimited.  Every GPU on which the library is
+ *    loaded carries the 2 MiB array until the process exits, whether or not this function is used.
+ *  - First use on a device looks up the array's device address (one runtime query, cached per
+ *    device).  Make that first call with the intended device current and before starting any stream
+ *    capture; later calls do no set-up.
+ *  - All calls share the one array.  Nothing in it needs clearing between calls (every partial that
+ *    is read has been written by the same call), but two calls that can run at the same time on the
+ *    GPU - different streams, or different host threads - would overwrite each other's partial sums:
+ *    keep calls to this function ordered with respect to each other.
+ *  - dY and dbias are device pointers of type `dtype`; the work is enqueued on `cuda_stream`. */
+lrd_status_t lrd_bias_grad_noalloc(const void* dY, int64_t ldy, int64_t M, int64_t N, void* dbias,
+                                   lrd_dtype_t dtype, void* cuda_stream);
 
 /* ---- Tucker-2 decomposed 3x3 convolution (Eq. 4, Fig. 1) -------------------------------- */
 

@@ -17,7 +17,7 @@ _lib = C.CDLL(LIB_PATH)
 
 # enums -------------------------------------------------------------------------------------------
 (LRD_OK, LRD_ERR_INVALID_ARG, LRD_ERR_BAD_RANK, LRD_ERR_ALIGNMENT, LRD_ERR_WORKSPACE, LRD_ERR_UNSUPPORTED,
- LRD_ERR_ARCH, LRD_ERR_CUDA, LRD_ERR_TIMEOUT) = range(9)
+ LRD_ERR_ARCH, LRD_ERR_CUDA, LRD_ERR_TIMEOUT, LRD_ERR_TOO_LARGE) = range(10)
 LRD_F32, LRD_BF16 = 0, 1
 LRD_FREEZE_NONE, LRD_FREEZE_U, LRD_FREEZE_V = 0, 1, 2
 LRD_TK_FREEZE_NONE, LRD_TK_FREEZE_FACTORS, LRD_TK_FREEZE_CORE = 0, 1, 2
@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc",
 ]
 
 
@@ -72,6 +72,8 @@ _lib.lrd_dense_fwd.restype = _int
 _lib.lrd_dense_fwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 4 + [_vp, _sz, _vp]
 _lib.lrd_dense_bwd.restype = _int
 _lib.lrd_dense_bwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 6 + [_vp, _sz, _vp]
+_lib.lrd_bias_grad_noalloc.restype = _int
+_lib.lrd_bias_grad_noalloc.argtypes = [_vp, _i64, _i64, _i64, _vp, _int, _vp]
 _lib.lrd_tucker2_fwd.restype = _int
 _lib.lrd_tucker2_fwd.argtypes = [C.POINTER(lrd_tucker2_desc_t)] + [_vp] * 8 + [_int, _vp, _sz, _vp]
 _lib.lrd_tucker2_bwd.restype = _int
@@ -210,6 +212,14 @@ def lrd_tucker2_bwd(desc, dY, X, A, G, Bm, Z1_save, Z2_save, dX, dA, dG, dB, dbi
     st = _lib.lrd_tucker2_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(A), _ptr(G), _ptr(Bm), _ptr(Z1_save),
                               _ptr(Z2_save), _ptr(dX), _ptr(dA), _ptr(dG), _ptr(dB), _ptr(dbias), freeze, w, n,
                               _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_bias_grad_noalloc(dY, ldy, M, N, dbias, dtype, stream=None, check=True):
+    """Column sums of dY into dbias with the library's built-in scratch (no workspace, no allocation)."""
+    st = _lib.lrd_bias_grad_noalloc(_ptr(dY), ldy, M, N, _ptr(dbias), dtype, _stream(stream))
     if check:
         _check(st)
     return st

@@ -161,6 +161,7 @@ const char* lrd_status_string(lrd_status_t s) {
         case LRD_ERR_ARCH: return "device is not sm_100";
         case LRD_ERR_CUDA: return "CUDA call failed";
         case LRD_ERR_TIMEOUT: return "device-side wait timed out";
+        case LRD_ERR_TOO_LARGE: return "size exceeds the fixed limit of this entry point";
     }
     return "unknown status";
 }

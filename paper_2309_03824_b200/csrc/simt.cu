@@ -300,3 +300,58 @@ lrd_status_t simt_colsum(const void* A, int64_t lda, int64_t M, int64_t N, void*
 }
 
 }  // namespace lrd
+
+// ---- bias gradient without any caller-provided or allocated scratch -----------------------------------
+// The partial column sums of the two-stage kernels live in a file-scope device array, so a caller
+// that may not allocate device memory can still get the many-block version.
+namespace {
+
+constexpr int64_t kNoAllocMaxN = 8192;                           // widest dY this entry point accepts
+constexpr int kNoAllocMaxSplits = 64;
+constexpr size_t kNoAllocFloats = (size_t)kNoAllocMaxN * kNoAllocMaxSplits;   // 2 MiB per GPU that loads the library
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_noalloc_ptr[kMaxDevices] = {};                          // device address of the array, per device
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a kernel can use:
+// the device address is asked for once per device (with that device current) and cached.
+lrd_status_t noalloc_scratch(float** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LRD_ERR_CUDA;
+    if (!g_noalloc_ptr[dev]) {
+        float* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return LRD_ERR_CUDA;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return LRD_OK;
+}
+
+}  // namespace
+
+extern "C" lrd_status_t lrd_bias_grad_noalloc(const void* dY, int64_t ldy, int64_t M, int64_t N, void* dbias,
+                                              lrd_dtype_t dtype, void* cuda_stream) {
+    if (M < 0 || N < 1 || (dtype != LRD_F32 && dtype != LRD_BF16)) return LRD_ERR_INVALID_ARG;
+    if (!dbias || (M > 0 && !dY)) return LRD_ERR_INVALID_ARG;
+    if (ldy == 0) ldy = N;
+    if (ldy < N) return LRD_ERR_INVALID_ARG;
+    if (N > kNoAllocMaxN) return LRD_ERR_TOO_LARGE;
+    const size_t e = lrd::elem_size(dtype);
+    if (((uintptr_t)dbias % e) || ((uintptr_t)dY % e)) return LRD_ERR_ALIGNMENT;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return LRD_ERR_CUDA;
+    if (major != 10) return LRD_ERR_ARCH;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (M == 0) return cudaMemsetAsync(dbias, 0, (size_t)N * e, stream) == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+    float* scratch = nullptr;
+    const lrd_status_t st = noalloc_scratch(&scratch);
+    if (st != LRD_OK) return st;
+    // Same kernels and same row split as the workspace path (splits <= 64, so the partial sums fit);
+    // stage 1 writes every partial that stage 2 reads, so nothing left by an earlier call is ever used.
+    const int splits = lrd::colsum_splits(M);
+    return dtype == LRD_F32 ? lrd::colsum_two_stage_t<float>(dY, ldy, M, N, dbias, scratch, splits, stream)
+                            : lrd::colsum_two_stage_t<__nv_bfloat16>(dY, ldy, M, N, dbias, scratch, splits, stream);
+}

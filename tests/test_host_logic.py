@@ -52,7 +52,7 @@ def test_freeze_schedule_and_plan_bit_exact_against_oracle():
 
 
 def test_status_strings_and_workspace_queries():
-    for s in range(9):
+    for s in range(10):
         assert b.lrd_status_string(s) and b.lrd_status_string(s) != "unknown status"
     assert b.lrd_status_string(99) == "unknown status"
     d = b.linear_desc(4096, 768, 768, 192, b.LRD_BF16)

@@ -29,6 +29,8 @@ size_t split_bytes(const Tk& t) {
         const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P), b = tc_split_workspace_bytes(t.C, t.r1, t.P);
         need = need > a ? need : a;
         need = need > b ? need : b;
+        const size_t f = tc_conv_filter_scratch_bytes(t.B, t.H, t.W, t.r1, t.r2);
+        need = need > f ? need : f;
     }
     return need;
 }
@@ -100,24 +102,29 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
         LRD_TRY(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, partials, pbytes, s));
         if (dbias) LRD_TRY(colsum(dY, t.S, t.P, t.S, dbias, t.dt, partials, pbytes, s));
     }
-    if (core) LRD_TRY(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    if (core) LRD_TRY(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, partials, pbytes, s));
     return LRD_OK;
 }
 
-// Core convolution dispatch: the general kernels for now serve every shape.
+// Core convolution dispatch: tensor-core implicit GEMM where the geometry qualifies, else the general kernels.
 lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
                          int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
-    (void)path;
+    if (path != LRD_PATH_GENERAL && tc_conv_eligible(B, H, W, ci, co, dt, in, G, out))
+        return tc_conv3x3(false, in, G, out, B, H, W, ci, co, s);
     return simt_conv3x3_fwd(in, G, out, B, H, W, ci, co, dt, s);
 }
 lrd_status_t conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W, int64_t ci,
                               int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
-    (void)path;
+    if (path != LRD_PATH_GENERAL && tc_conv_eligible(B, H, W, ci, co, dt, dout, G, din))
+        return tc_conv3x3(true, dout, G, din, B, H, W, ci, co, s);
     return simt_conv3x3_bwd_data(dout, G, din, B, H, W, ci, co, dt, s);
 }
 lrd_status_t conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
-                                int64_t ci, int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
-    (void)path;
+                                int64_t ci, int64_t co, lrd_dtype_t dt, int path, float* scratch, size_t scratch_bytes,
+                                cudaStream_t s) {
+    if (path != LRD_PATH_GENERAL && tc_conv_eligible(B, H, W, ci, co, dt, dout, in, dG) &&
+        scratch_bytes >= tc_conv_filter_scratch_bytes(B, H, W, ci, co))
+        return tc_conv3x3_filter(dout, in, dG, B, H, W, ci, co, scratch, scratch_bytes, s);
     return simt_conv3x3_bwd_filter(dout, in, dG, B, H, W, ci, co, dt, s);
 }
 

@@ -25,12 +25,22 @@ lrd_status_t simt_conv3x3_bwd_data(const void* dout, const void* G, void* din, i
 lrd_status_t simt_conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
                                      int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s);
 
+// Tensor-core 3x3 core (bf16, W <= 128, channel counts multiples of 8, 16-byte aligned bases).
+bool tc_conv_eligible(int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, lrd_dtype_t dt, const void* p0,
+                      const void* p1, const void* p2);
+size_t tc_conv_filter_scratch_bytes(int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co);
+lrd_status_t tc_conv3x3(bool dgrad, const void* img, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
+                        int64_t co, cudaStream_t s);
+lrd_status_t tc_conv3x3_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W, int64_t ci,
+                               int64_t co, float* scratch, size_t scratch_bytes, cudaStream_t s);
+
 // Path dispatch for the core (tensor-core kernel where the shape qualifies, else general).
 lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
                          int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
 lrd_status_t conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W, int64_t ci,
                               int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
 lrd_status_t conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
-                                int64_t ci, int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
+                                int64_t ci, int64_t co, lrd_dtype_t dt, int path, float* scratch, size_t scratch_bytes,
+                                cudaStream_t s);
 
 }  // namespace lrd

@@ -119,6 +119,22 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(ms, world, device):
+    """A timing in ms -> the slowest rank's (all-reduce MAX over the process group); identity for one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank, world, ms_per_step):
+    """Weak scaling: every rank runs the same workload; throughput counts all ranks' tokens over the slowest rank's time."""
+    return tokens_per_rank * world / (ms_per_step * 1e-3)
+
+
 # ---- the oracle, timed (CPU baseline / reference arm) ------------------------------------------------
 def oracle_block_seconds(layers_np, min_seconds, max_reps=400):
     """Forward + backward of the whole block in the fp64 oracle, alternating masks; returns
@@ -324,11 +340,7 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         t1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
         barrier()
         return ms, t0, t1
 
@@ -342,7 +354,7 @@ def main():
     clocks = sampler.summary(t0, t1) if rank == 0 else None
     ms_per_step = ms / args.steps
     tokens = wl.C1_M * world
-    value = tokens / (ms_per_step * 1e-3)
+    value = whole_job_value(wl.C1_M, world, ms_per_step)
 
     # ---- end to end: activations from pinned host memory in, weight gradients out, every step ------
     h2d = sum(L["hX"].numel() * 2 + L["hdY"].numel() * 2 for L in layers)

@@ -156,6 +156,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         int s = 0;
         bool ok = true;
         const uint32_t idesc1 = idesc_bf16(p.RS, false, true);
+        const uint64_t a_desc0 = smem_desc_sw128(0, 0, 1024);
+        const uint64_t b_desc0 = smem_desc(0, p_box_bytes, 8u * p.swb, p.swb);
         for (int g = 0; g < ng1; ++g) {
             ok = !pair_sync_or(false) && ok;
             if (lane == 0 && ok) {
@@ -163,14 +165,16 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 const uint32_t in_src = ring_base + s * p.stage1_bytes;
                 const uint32_t p_src = in_src + p.G1 * kInTileBytes;
                 const int nkb = min(p.G1, p.kb1 - g * p.G1);
+                // descriptors differ only in the start-address field (bits 0-13, in 16-byte units): build one
+                // per operand and add offsets
+                uint64_t ad = a_desc0 + ((in_src >> 4) & 0x3FFFu);
+                uint64_t bd = b_desc0 + ((p_src >> 4) & 0x3FFFu);
                 for (int i = 0; i < nkb; ++i) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t ad = smem_desc_sw128(in_src + i * kInTileBytes + kk * 32, 0, 1024);
-                        const uint64_t bd = smem_desc(p_src + (uint32_t)(i * 64 + kk * 16) * (uint32_t)p.swb, p_box_bytes,
-                                                      8u * p.swb, p.swb);
-                        mma_bf16_ss(tmem_base, ad, bd, idesc1, (g > 0 || i > 0 || kk > 0) ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_bf16_ss(tmem_base, ad + 2u * kk, bd + (uint64_t)(kk * p.swb), idesc1, (g > 0 || i > 0 || kk > 0) ? 1u : 0u);
+                    ad += kInTileBytes >> 4;
+                    bd += (uint64_t)(4 * p.swb);              // 64 rows of swb bytes
                 }
                 mma_commit(smem_u32(&empty1[s]));
             }
@@ -178,6 +182,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         }
         if (lane == 0 && ok) mma_commit(smem_u32(&tacc_bar));
         const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
+        const uint64_t t_desc0 = smem_desc(t_base, 0, 8u * t_sw, t_sw);
         s = 0;
         int i2 = 0;
         for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
@@ -189,16 +194,16 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                     tc_fence_after();
                     const uint32_t q_src = ring_base + s * p.stage2_bytes;
                     const int nkb = min(p.G2, p.kb2 - g * p.G2);
+                    uint64_t bd = a_desc0 + ((q_src >> 4) & 0x3FFFu);
                     for (int i = 0; i < nkb; ++i) {
                         const int kb = g * p.G2 + i;
                         const int nks = min(4, p.ks2 - kb * 4);
                         for (int kk = 0; kk < nks; ++kk) {
                             const int ks = kb * 4 + kk;                       // 16-column step within T
-                            const uint64_t ad = smem_desc(t_base + (uint32_t)(ks / t_steps) * t_atom_bytes + (uint32_t)(ks % t_steps) * 32u,
-                                                          0, 8u * t_sw, t_sw);
-                            const uint64_t bd = smem_desc_sw128(q_src + i * q_tile_bytes + kk * 32, 0, 1024);
-                            mma_bf16_ss(d_tmem, ad, bd, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
+                            const uint64_t ad = t_desc0 + (((uint32_t)(ks / t_steps) * t_atom_bytes + (uint32_t)(ks % t_steps) * 32u) >> 4);
+                            mma_bf16_ss(d_tmem, ad, bd + 2u * kk, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
                         }
+                        bd += q_tile_bytes >> 4;
                     }
                     mma_commit(smem_u32(&empty2[s]));
                     if (g == ng2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));

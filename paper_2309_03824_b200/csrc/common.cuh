@@ -22,6 +22,8 @@ struct GemmArgs {
     const void* B; int64_t ldb; bool b_mn_major;
     void* C; int64_t ldc;
     const void* bias;          // [N] or nullptr, same dtype as C
+    void* a_colsum = nullptr;  // optional [M]: sum over k of A(m, k) (the bias gradient when A is dY); only on the
+                               // tensor-core path with both operands MN-major, see tc_gemm_colsum_ok()
     lrd_dtype_t dtype;         // storage type of A, B, C, bias
 };
 

@@ -98,9 +98,15 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
     if (dX || factors) LRD_TRY(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
     if (dX) LRD_TRY(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
     if (factors) {
-        LRD_TRY(run_gemm(make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt), path, true, partials, pbytes, s));
+        GemmArgs gb = make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt);
+        bool db_done = false;
+        if (dbias && path != LRD_PATH_GENERAL) {          // the bias gradient rides on the dB product (A = dY)
+            gb.a_colsum = dbias;
+            if (tc_gemm_colsum_ok(gb)) db_done = true; else gb.a_colsum = nullptr;
+        }
+        LRD_TRY(run_gemm(gb, path, true, partials, pbytes, s));
         LRD_TRY(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, partials, pbytes, s));
-        if (dbias) LRD_TRY(colsum(dY, t.S, t.P, t.S, dbias, t.dt, partials, pbytes, s));
+        if (dbias && !db_done) LRD_TRY(colsum(dY, t.S, t.P, t.S, dbias, t.dt, partials, pbytes, s));
     }
     if (core) LRD_TRY(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, partials, pbytes, s));
     return LRD_OK;

@@ -283,9 +283,14 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
             LRD_TRY(run_gemm(gemm(L.M, L.K, L.r, dZ, L.r, false, V, L.ldv, false, dX, L.ldx, nullptr, L.dt), false, nullptr, 0, s));
     }
     if (plan & LRD_PLAN_DU) {
-        LRD_TRY(run_gemm(gemm(L.N, L.r, L.M, dY, L.ldy, true, Z_save, L.ldz, true, dU, L.ldu, nullptr, L.dt), true, partials,
-                         partial_bytes, s));
-        if (dbias) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, partial_bytes, s));
+        GemmArgs gu = gemm(L.N, L.r, L.M, dY, L.ldy, true, Z_save, L.ldz, true, dU, L.ldu, nullptr, L.dt);
+        bool db_done = false;
+        if (dbias && g_path.load() != LRD_PATH_GENERAL) {      // db rides on the dU product (A = dY): no second pass over dY
+            gu.a_colsum = dbias;
+            if (tc_gemm_colsum_ok(gu)) db_done = true; else gu.a_colsum = nullptr;
+        }
+        LRD_TRY(run_gemm(gu, true, partials, partial_bytes, s));
+        if (dbias && !db_done) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, partial_bytes, s));
     }
     if (plan & LRD_PLAN_DV)
         LRD_TRY(run_gemm(gemm(L.K, L.r, L.M, X, L.ldx, true, dZ, L.r, true, dV, L.ldv, nullptr, L.dt), true, partials,
@@ -318,9 +323,14 @@ lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const 
     }
     float* partials = (float*)((uint8_t*)workspace + 256);
     if (dX) LRD_TRY(run_gemm(gemm(L.M, L.K, L.N, dY, L.ldy, false, W, L.ldv, true, dX, L.ldx, nullptr, L.dt), false, nullptr, 0, s));
-    LRD_TRY(run_gemm(gemm(L.N, L.K, L.M, dY, L.ldy, true, X, L.ldx, true, dW, L.ldv, nullptr, L.dt), true, partials,
-                     workspace_bytes - 256, s));
-    if (dbias) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, workspace_bytes - 256, s));
+    GemmArgs gw = gemm(L.N, L.K, L.M, dY, L.ldy, true, X, L.ldx, true, dW, L.ldv, nullptr, L.dt);
+    bool db_done = false;
+    if (dbias && g_path.load() != LRD_PATH_GENERAL) {
+        gw.a_colsum = dbias;
+        if (tc_gemm_colsum_ok(gw)) db_done = true; else gw.a_colsum = nullptr;
+    }
+    LRD_TRY(run_gemm(gw, true, partials, workspace_bytes - 256, s));
+    if (dbias && !db_done) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, workspace_bytes - 256, s));
     return LRD_OK;
 }
 

@@ -12,6 +12,8 @@ int tc_pick_bn(int64_t M, int64_t N);
 int tc_pick_splits(int64_t M, int64_t N, int64_t K);
 // fp32 partial-tile scratch a split product of this shape needs (0 when it is not split).
 size_t tc_split_workspace_bytes(int64_t M, int64_t N, int64_t K);
+// True when tc_gemm can also deliver g.a_colsum for this product (bf16, both operands MN-major, aligned).
+bool tc_gemm_colsum_ok(const GemmArgs& g);
 // allow_split: the reduction dimension may be split over blocks (weight gradients).
 lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes, cudaStream_t stream);
 

@@ -24,12 +24,16 @@ constexpr int BM = 128, BK = 64;
 constexpr int kThreads = 224;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
 
-template <int BN> struct Cfg {
-    static constexpr uint32_t B_STAGE_BYTES = BN * BK * 2;
+// ONES: every stage carries one more 64-wide MN-major block of B that holds 1.0 everywhere and is never
+// overwritten; with N = BN + 16 the MMA then also forms sum_k A(m, k) in accumulator column BN (the bias
+// gradient falls out of the dU product: its A operand is dY).
+template <int BN, bool ONES = false> struct Cfg {
+    static constexpr uint32_t B_STAGE_BYTES = BN * BK * 2 + (ONES ? 8192 : 0);
     static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 192 ? 5 : (BN >= 128 ? 6 : 8));
+    static constexpr int STAGES_RAW = (200 * 1024) / STAGE_BYTES;
+    static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
     static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack for 1024-B alignment
-    static constexpr uint32_t TMEM_COLS = BN <= 64 ? 64 : (BN <= 128 ? 128 : 256);
+    static constexpr uint32_t TMEM_COLS = (BN + (ONES ? 32 : 0)) <= 64 ? 64 : ((BN + (ONES ? 32 : 0)) <= 128 ? 128 : 256);
 };
 
 struct TcParams {
@@ -40,13 +44,16 @@ struct TcParams {
     int64_t ldc;
     const __nv_bfloat16* bias;
     int partial;        // 1: write fp32 partials
+    float* colsum_partial;        // ONES, split: [splits][M] partial sums over k of A
+    __nv_bfloat16* colsum_out;    // ONES, not split: [M]
     unsigned int* timeout_flag;
 };
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, bool ONES = false>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
-    using C = Cfg<BN>;
+    static_assert(!ONES || (A_MN && B_MN && BN <= 192), "the ones block rides on an MN-major B of at most 192 columns");
+    using C = Cfg<BN, ONES>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
@@ -71,6 +78,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         mbar_init(smem_u32(&acc_bar), 1);
         fence_mbar_init();
     }
+    if (ONES) {          // bf16 1.0 in every element of the extra block of each stage
+        for (uint32_t off = threadIdx.x * 16u; off < STAGES * 8192u; off += kThreads * 16u)
+            st_shared_v4(smem_base + (off / 8192u) * C::STAGE_BYTES + A_STAGE_BYTES + BN * 128u + (off % 8192u), 0x3F803F80u,
+                         0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+        fence_proxy_async_smem();
+    }
     if (warp == 1) {
         tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS);
         tmem_relinquish();
@@ -88,7 +101,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t ph = (it / STAGES) & 1;
                 if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, ab)) break;
                 const uint32_t fb = smem_u32(&full_bar[s]);
-                mbar_expect_tx(fb, C::STAGE_BYTES);
+                mbar_expect_tx(fb, A_STAGE_BYTES + BN * BK * 2);
                 const uint32_t a_dst = smem_base + s * C::STAGE_BYTES;
                 const uint32_t b_dst = a_dst + A_STAGE_BYTES;
                 const int k0 = kb * BK;
@@ -110,7 +123,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // MMA issuer.  It never waits on a barrier itself (a shared-memory read behind a tcgen05.commit
         // stalls until the committed MMAs finish): warp 6 waits and hands each ready stage over.
-        constexpr uint32_t idesc = idesc_bf16(BN, A_MN, B_MN);
+        const uint32_t idesc = idesc_bf16(BN + ((ONES && blockIdx.x == 0) ? 16 : 0), A_MN, B_MN);
         int s = 0;
         bool ok = true;
         for (int kb = kb_begin; kb < kb_end; ++kb) {
@@ -151,6 +164,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int64_t row = (int64_t)m0 + quarter * 32 + lane;
             const bool row_ok = row < p.M;
             const bool bias_vec_ok = p.bias && (((uintptr_t)p.bias & 15u) == 0);
+            if (ONES && blockIdx.x == 0) {                 // accumulator column BN = sum over k of A(row, k)
+                uint32_t cs[16];
+                tmem_ld_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + BN, cs);
+                tmem_ld_wait();
+                if (row_ok) {
+                    if (p.partial) p.colsum_partial[(int64_t)blockIdx.z * p.M + row] = __uint_as_float(cs[0]);
+                    else if (p.colsum_out) p.colsum_out[row] = __float2bfloat16_rn(__uint_as_float(cs[0]));
+                }
+            }
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
@@ -218,10 +240,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t M,
                                                             int64_t N, int64_t ldp,
                                                             const __nv_bfloat16* __restrict__ bias,
-                                                            __nv_bfloat16* __restrict__ C, int64_t ldc) {
+                                                            __nv_bfloat16* __restrict__ C, int64_t ldc,
+                                                            const float* __restrict__ colsum_partial,
+                                                            __nv_bfloat16* __restrict__ colsum_out) {
     const int64_t n4 = (N + 3) / 4;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= M * n4) return;
+    if (idx >= M * n4) {                                // trailing threads: the column sums, one row each
+        const int64_t m = idx - M * n4;
+        if (colsum_out && m < M) {
+            float t = 0.f;
+            for (int z = 0; z < splits; ++z) t += colsum_partial[(int64_t)z * M + m];
+            colsum_out[m] = __float2bfloat16_rn(t);
+        }
+        return;
+    }
     const int64_t m = idx / n4, n = (idx % n4) * 4;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const bool full = n + 4 <= N;
@@ -243,16 +275,16 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
         }
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, bool ONES = false>
 lrd_status_t launch(const CUtensorMap& tA, const CUtensorMap& tB, const TcParams& p, dim3 grid, cudaStream_t stream) {
-    auto kern = tc_gemm_kernel<BN, A_MN, B_MN>;
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, ONES>;
     static bool configured = false;     // per instantiation; the attribute is sticky per function
     if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN, ONES>::SMEM_BYTES) != cudaSuccess)
             return LRD_ERR_CUDA;
         configured = true;
     }
-    kern<<<grid, kThreads, Cfg<BN>::SMEM_BYTES, stream>>>(tA, tB, p);
+    kern<<<grid, kThreads, Cfg<BN, ONES>::SMEM_BYTES, stream>>>(tA, tB, p);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
@@ -312,18 +344,28 @@ int tc_pick_splits(int64_t M, int64_t N, int64_t K) {
     return (int)s;
 }
 
+// fp32 partial tiles [splits][M][ldp], then (for the optional column sums) [splits][M]
 size_t tc_split_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     const int s = tc_pick_splits(M, N, K);
-    return s > 1 ? align_up((size_t)s * M * ((N + 3) / 4 * 4) * sizeof(float), 256) : 0;
+    return s > 1 ? align_up((size_t)s * M * ((N + 3) / 4 * 4) * sizeof(float), 256) + align_up((size_t)s * M * sizeof(float), 256) : 0;
+}
+
+bool tc_gemm_colsum_ok(const GemmArgs& g) {
+    return tc_gemm_eligible(g) && g.a_mn_major && g.b_mn_major && (((uintptr_t)g.a_colsum & 1u) == 0);
 }
 
 lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes,
                      cudaStream_t stream) {
     if (!tc_gemm_eligible(g)) return LRD_ERR_UNSUPPORTED;
     int splits = allow_split ? tc_pick_splits(g.M, g.N, g.K) : 1;
-    const int bn = pick_bn(g.M, g.N, splits > 1);
+    int bn = pick_bn(g.M, g.N, splits > 1);
+    const bool ones = g.a_colsum != nullptr;
+    if (ones && !tc_gemm_colsum_ok(g)) return LRD_ERR_UNSUPPORTED;
+    if (ones && bn > 192) bn = 192;                    // the ones block needs 16 accumulator columns beside the tile
     const int64_t ldp = (g.N + 3) / 4 * 4;
-    if (splits > 1 && (!partials || partial_bytes < (size_t)splits * g.M * ldp * sizeof(float))) return LRD_ERR_WORKSPACE;
+    const size_t tile_bytes = align_up((size_t)splits * g.M * ldp * sizeof(float), 256);
+    if (splits > 1 && (!partials || partial_bytes < tile_bytes + (ones ? (size_t)splits * g.M * sizeof(float) : 0)))
+        return LRD_ERR_WORKSPACE;
     const int kb_total = (int)((g.K + BK - 1) / BK);
     const int kb_per = (kb_total + splits - 1) / splits;
 
@@ -341,8 +383,17 @@ lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_
     p.C = splits > 1 ? (void*)partials : g.C;
     p.ldc = g.ldc;
     p.bias = splits > 1 ? nullptr : (const __nv_bfloat16*)g.bias;
+    p.colsum_partial = (ones && splits > 1) ? (float*)((uint8_t*)partials + tile_bytes) : nullptr;
+    p.colsum_out = (ones && splits == 1) ? (__nv_bfloat16*)g.a_colsum : nullptr;
     dim3 grid((unsigned)((g.N + bn - 1) / bn), (unsigned)((g.M + BM - 1) / BM), (unsigned)splits);
     lrd_status_t st;
+    if (ones) {
+        switch (bn) {
+            case 192: st = launch<192, true, true, true>(tA, tB, p, grid, stream); break;
+            case 128: st = launch<128, true, true, true>(tA, tB, p, grid, stream); break;
+            default:  st = launch<64, true, true, true>(tA, tB, p, grid, stream); break;
+        }
+    } else
     switch (bn) {
         case 256: st = launch_major<256>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
         case 192: st = launch_major<192>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
@@ -350,9 +401,10 @@ lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_
         default:  st = launch_major<64>(g.a_mn_major, g.b_mn_major, tA, tB, p, grid, stream); break;
     }
     if (st != LRD_OK || splits == 1) return st;
-    const int64_t work = g.M * ((g.N + 3) / 4);
+    const int64_t work = g.M * ((g.N + 3) / 4) + (ones ? g.M : 0);
     splitk_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(
-        partials, splits, g.M, g.N, ldp, (const __nv_bfloat16*)g.bias, (__nv_bfloat16*)g.C, g.ldc);
+        partials, splits, g.M, g.N, ldp, (const __nv_bfloat16*)g.bias, (__nv_bfloat16*)g.C, g.ldc, p.colsum_partial,
+        ones ? (__nv_bfloat16*)g.a_colsum : nullptr);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }

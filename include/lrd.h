@@ -114,6 +114,13 @@ const char* lrd_status_string(lrd_status_t s);
  * for an unknown value.  Not thread-safe against concurrent launches. */
 lrd_status_t lrd_set_path(lrd_path_t path);
 
+/* Launch-shape overrides of the fused chain kernel, for measurement sweeps (no counterpart in the
+ * paper): blocks per cluster (1, 2 or 4), 64-deep k-blocks per pipeline stage of the first product
+ * (1..4), column-chunk width of the second product (128, 192 or 256).  0 = automatic (the default).
+ * A shape the override makes infeasible falls back to the unfused products.  Process-wide, not
+ * thread-safe against concurrent launches.  Returns LRD_ERR_INVALID_ARG for values outside the lists. */
+lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chunk_columns);
+
 /* Synchronises the current device, then reports and clears the device-side timeout flag:
  * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
 lrd_status_t lrd_check_device_status(void);

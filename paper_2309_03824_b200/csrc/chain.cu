@@ -2,44 +2,49 @@
 //
 // A cluster of C blocks owns one 128-row tile.
 //   Phase 1  block c forms its r/C-column slice of T = In P in tensor memory (TMA-fed tcgen05.mma:
-//            In K-major, the slice of P MN-major).
+//            In K-major, the slice of P MN-major).  The whole dynamic shared memory is the ring of
+//            this phase: many small stages, so that nearly all of it is in flight at any time.
 //   Gather   four warps read the slice (tcgen05.ld), round it to bf16 and write it into this block's T
 //            buffer (K-major, swizzled, slices are whole atoms = one contiguous range); one thread then
 //            copies the range into every peer's T buffer with bulk DSMEM copies that complete on the
-//            peer's barrier.  T never goes to global memory unless T_save asks.
-//   Phase 2  block c forms every C-th column chunk of Out = T Q^T (T from shared memory, Q by TMA),
-//            double-buffered in tensor memory; the epilogue adds the bias, rounds to bf16 and writes
-//            through shared memory with TMA stores (which clip the ragged edges).
-// A pipeline stage holds a GROUP of 64-deep k-blocks behind one barrier pair: the cost of a stage
-// turn-around (barrier round trip, hand-over to the MMA thread, TMA issue) is per stage, not per byte,
-// so stages are made as large as shared memory allows.  The two phases lay their stages out
-// differently over the same ring.
+//            peer's barrier.  The T buffer lies over ring space of phase 1, so a block pushes only after
+//            every block of the cluster has reported the end of its phase-1 MMAs.  T never goes to
+//            global memory unless T_save asks.
+//   Phase 2  block c forms every C-th column chunk of Out = T Q^T (T from shared memory, Q by TMA, one
+//            64-deep tile per stage), double-buffered in tensor memory; the epilogue adds the bias,
+//            rounds to bf16 and leaves through [128 x 64] shared-memory slabs by TMA stores (which
+//            clip the ragged edges).
 // Warp 0: TMA producer.  Warp 1: tensor memory + MMA issue.  Warps 2-5: gather and epilogue.
-// Warp 6: waits on the stage barriers for warp 1 and hands ready stages over by a named barrier (the
-// issuing thread must not read shared memory behind a tcgen05.commit: that read waits for the MMAs).
+// Every wait is bounded; a wait that runs out raises the device timeout flag and the block tears
+// down in order.
 #include "chain.cuh"
 
 #include "ptx.cuh"
 #include "tc.cuh"
 #include "tma.cuh"
 
+#ifndef LRD_TS
+#define LRD_TS(slot)      // timestamp hook of profiling builds (one thread, clock counter into a trace buffer); compiled out
+#endif
+
 namespace lrd {
 namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 224;
-constexpr int kMaxStages = 8;
-constexpr uint32_t kSmemLimit = 226 * 1024;         // dynamic shared memory; the rest is left for the barriers
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 12;
+constexpr uint32_t kSmemLimit = 224 * 1024;         // dynamic shared memory; the rest is left for the barriers and the bias
 constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile of one k-block: 128 rows x 64 k
-constexpr uint32_t kSlabBytes = 32 * 64;            // epilogue slab: 32 rows x 32 columns of bf16
-constexpr uint32_t kStagingBytes = 4 * 2 * kSlabBytes;
+constexpr uint32_t kSlabBytes = 128 * 64 * 2;       // epilogue slab: 128 rows x 64 columns of bf16
+constexpr uint32_t kStagingBytes = 2 * kSlabBytes;
 
 struct ChainParams {
     int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, N2;
-    int G1, S1, G2, S2;       // k-blocks per stage and stage count of phase 1 / phase 2
+    int G1, S1, S2;           // k-blocks per phase-1 stage; stage counts of the two phases
     uint32_t stage1_bytes, stage2_bytes, t_bytes;
     int taw;                  // columns per atom of the T buffer (64, 32 or 16; swizzle span = 2 * taw bytes)
+    int t_steps_lg;           // log2 of the MMA k-steps (16 columns) per atom
     const __nv_bfloat16* bias;
     int has_tsave;
     unsigned int* timeout_flag;
@@ -52,25 +57,31 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages],
         tacc_bar, tready_bar, out_full[2], out_empty[2];
+    __shared__ __align__(16) float bias_s[2][256];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
+    // phase 1: [T | ring of S1 stages];  phase 2: [T | two output slabs | ring of S2 stages]
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t t_base = smem_base;
-    const uint32_t staging_base = t_base + p.t_bytes;
-    const uint32_t ring_base = staging_base + kStagingBytes;
+    const uint32_t ring1_base = t_base + p.t_bytes;
+    const uint32_t staging_base = ring1_base;
+    const uint32_t ring2_base = staging_base + kStagingBytes;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
     const uint32_t t_sw = 2u * (uint32_t)p.taw, t_atom_bytes = 128u * t_sw;   // T: atoms of [128 rows x taw columns]
-    const int t_steps = p.taw / 16;                                           // MMA k-steps per atom
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    // The warp index is made provably warp-uniform, and the single-thread instructions (TMA, MMA, commit)
+    // are issued under elect.sync by an otherwise converged warp: their operands then stay in uniform
+    // registers.  (Issued from a lane-0 branch instead, every such instruction costs hundreds of cycles.)
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0);
+    const int lane = threadIdx.x % 32;
     const int c = (int)cluster_ctarank();
     const int m0 = blockIdx.y * 128;
-    const int ng1 = (p.kb1 + p.G1 - 1) / p.G1, ng2 = (p.kb2 + p.G2 - 1) / p.G2;   // stage turns per phase / chunk
+    const int ng1 = (p.kb1 + p.G1 - 1) / p.G1;                                 // stage turns of phase 1
     // phase-1 stage: G1 In tiles, then the P boxes (one per column atom, 64 G1 rows tall)
     const uint32_t p_box_bytes = 64u * (uint32_t)p.G1 * (uint32_t)p.swb;
-    const uint32_t q_tile_bytes = (uint32_t)p.BN2 * 128u;
 
     if (threadIdx.x == 0) {
+        LRD_TS(0);
         abort_flag = 0;
         prefetch_tmap(&tmIn);
         prefetch_tmap(&tmP);
@@ -98,14 +109,15 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     }
     tc_fence_before();
     __syncthreads();
-    cluster_arrive();          // every block's barriers exist before any peer touches them
-    cluster_wait();
+    // Cluster barrier 1 (every block's barriers exist before a peer pushes into it): arrive now, wait
+    // only where the first remote operation is near.  Until then a block touches its own memory only.
+    cluster_arrive();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    if (threadIdx.x == 0) { LRD_TS(1); }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        // Lane 0 waits for the stage and arms its barrier; then lane l issues copy l of the stage.
         int s = 0;
         uint32_t ph = 1;                                     // parity to wait on for an empty stage
         bool ok = true;
@@ -113,62 +125,63 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         const int n_pbox = p.RS / atom_cols;
         for (int g = 0; g < ng1 && ok; ++g) {
             const uint32_t fb = smem_u32(&full1[s]);
-            if (lane == 0) {
-                ok = mbar_wait(smem_u32(&empty1[s]), ph, ab);
-                if (ok) mbar_expect_tx(fb, p.stage1_bytes);
-            }
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            ok = mbar_wait_uniform(smem_u32(&empty1[s]), ph, ab);
             if (!ok) break;
-            const uint32_t dst = ring_base + s * p.stage1_bytes;
+            const uint32_t dst = ring1_base + s * p.stage1_bytes;
             const int kb0 = g * p.G1;
-            if (lane < p.G1)                                 // k-blocks past K1 read as zeros
-                tma_load_2d(dst + lane * kInTileBytes, &tmIn, fb, (kb0 + lane) * 64, m0);
-            else if (lane < p.G1 + n_pbox)
-                tma_load_2d(dst + p.G1 * kInTileBytes + (lane - p.G1) * p_box_bytes, &tmP, fb,
-                            c * p.RS + (lane - p.G1) * atom_cols, kb0 * 64);
+            if (elect_one()) {
+                if (g == 0) { LRD_TS(2); }
+                mbar_expect_tx(fb, p.stage1_bytes);
+                for (int i = 0; i < p.G1; ++i)               // k-blocks past K1 read as zeros
+                    tma_load_2d(dst + i * kInTileBytes, &tmIn, fb, (kb0 + i) * 64, m0);
+                for (int i = 0; i < n_pbox; ++i)
+                    tma_load_2d(dst + p.G1 * kInTileBytes + i * p_box_bytes, &tmP, fb, c * p.RS + i * atom_cols, kb0 * 64);
+            }
+            __syncwarp();
             if (++s == p.S1) { s = 0; ph ^= 1; }
         }
+        if (lane == 0) { LRD_TS(3); }
         // the ring is laid out anew for phase 2: wait until every phase-1 MMA has read its operands
-        if (lane == 0 && ok) ok = mbar_wait(smem_u32(&tacc_bar), 0, ab);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (ok) ok = mbar_wait_uniform(smem_u32(&tacc_bar), 0, ab);
+        if (lane == 0) { LRD_TS(4); }
         s = 0;
         ph = 1;
         for (int j = c; j < p.n_chunks && ok; j += p.C) {
-            for (int g = 0; g < ng2; ++g) {
+            for (int kb = 0; kb < p.kb2; ++kb) {             // columns past r read as zeros (never multiplied)
                 const uint32_t fb = smem_u32(&full2[s]);
-                if (lane == 0) {
-                    ok = mbar_wait(smem_u32(&empty2[s]), ph, ab);
-                    if (ok) mbar_expect_tx(fb, p.stage2_bytes);
-                }
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                ok = mbar_wait_uniform(smem_u32(&empty2[s]), ph, ab);
                 if (!ok) break;
-                if (lane < p.G2)                             // k-blocks past r read as zeros
-                    tma_load_2d(ring_base + s * p.stage2_bytes + lane * q_tile_bytes, &tmQ, fb, (g * p.G2 + lane) * 64,
-                                j * p.BN2);
+                if (elect_one()) {
+                    mbar_expect_tx(fb, p.stage2_bytes);
+                    tma_load_2d(ring2_base + s * p.stage2_bytes, &tmQ, fb, kb * 64, j * p.BN2);
+                }
+                __syncwarp();
                 if (++s == p.S2) { s = 0; ph ^= 1; }
             }
         }
-        __syncwarp();
+        if (lane == 0) { LRD_TS(5); }
+        cluster_wait();        // barrier 1
+        cluster_arrive();      // barrier 2
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // Never waits on a barrier itself: warp 6 does the waiting and hands each ready stage over
-        // through a named barrier.  Both warps run the same loops.
         int s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         const uint32_t idesc1 = idesc_bf16(p.RS, false, true);
         const uint64_t a_desc0 = smem_desc_sw128(0, 0, 1024);
         const uint64_t b_desc0 = smem_desc(0, p_box_bytes, 8u * p.swb, p.swb);
         for (int g = 0; g < ng1; ++g) {
-            ok = !pair_sync_or(false) && ok;
-            if (lane == 0 && ok) {
-                tc_fence_after();
-                const uint32_t in_src = ring_base + s * p.stage1_bytes;
-                const uint32_t p_src = in_src + p.G1 * kInTileBytes;
-                const int nkb = min(p.G1, p.kb1 - g * p.G1);
-                // descriptors differ only in the start-address field (bits 0-13, in 16-byte units): build one
-                // per operand and add offsets
-                uint64_t ad = a_desc0 + ((in_src >> 4) & 0x3FFFu);
-                uint64_t bd = b_desc0 + ((p_src >> 4) & 0x3FFFu);
+            ok = mbar_wait_uniform(smem_u32(&full1[s]), ph, ab);
+            if (!ok) break;
+            if (g == 0 && lane == 0) { LRD_TS(6); }
+            tc_fence_after();
+            const uint32_t in_src = ring1_base + s * p.stage1_bytes;
+            const uint32_t p_src = in_src + p.G1 * kInTileBytes;
+            const int nkb = min(p.G1, p.kb1 - g * p.G1);
+            // descriptors differ only in the start-address field (bits 0-13, in 16-byte units)
+            uint64_t ad = a_desc0 + ((in_src >> 4) & 0x3FFFu);
+            uint64_t bd = b_desc0 + ((p_src >> 4) & 0x3FFFu);
+            if (elect_one()) {
                 for (int i = 0; i < nkb; ++i) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
@@ -178,76 +191,59 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 }
                 mma_commit(smem_u32(&empty1[s]));
             }
-            if (++s == p.S1) s = 0;
+            __syncwarp();
+            if (++s == p.S1) { s = 0; ph ^= 1; }
         }
-        if (lane == 0 && ok) mma_commit(smem_u32(&tacc_bar));
+        if (ok && elect_one()) mma_commit(smem_u32(&tacc_bar));
+        __syncwarp();
+        if (lane == 0) { LRD_TS(7); }
+        // every slice of T has landed in this block's buffer (which also means the phase-1 accumulator
+        // columns have been read out)
+        if (ok) ok = mbar_wait_cluster_uniform(smem_u32(&tready_bar), 0, ab);
+        if (lane == 0) { LRD_TS(8); }
         const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
         const uint64_t t_desc0 = smem_desc(t_base, 0, 8u * t_sw, t_sw);
         s = 0;
-        int i2 = 0;
-        for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
-            const uint32_t d_tmem = tmem_base + (uint32_t)(i2 & 1) * 256u;
-            for (int g = 0; g < ng2; ++g) {
-                // (before a chunk's first stage warp 6 has also seen T complete and the accumulator buffer drained)
-                ok = !pair_sync_or(false) && ok;
-                if (lane == 0 && ok) {
-                    tc_fence_after();
-                    const uint32_t q_src = ring_base + s * p.stage2_bytes;
-                    const int nkb = min(p.G2, p.kb2 - g * p.G2);
-                    uint64_t bd = a_desc0 + ((q_src >> 4) & 0x3FFFu);
-                    for (int i = 0; i < nkb; ++i) {
-                        const int kb = g * p.G2 + i;
-                        const int nks = min(4, p.ks2 - kb * 4);
-                        for (int kk = 0; kk < nks; ++kk) {
-                            const int ks = kb * 4 + kk;                       // 16-column step within T
-                            const uint64_t ad = t_desc0 + (((uint32_t)(ks / t_steps) * t_atom_bytes + (uint32_t)(ks % t_steps) * 32u) >> 4);
-                            mma_bf16_ss(d_tmem, ad, bd + 2u * kk, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
-                        }
-                        bd += q_tile_bytes >> 4;
-                    }
-                    mma_commit(smem_u32(&empty2[s]));
-                    if (g == ng2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
-                }
-                if (++s == p.S2) s = 0;
-            }
-        }
-        __syncwarp();
-    } else if (warp == 6) {
-        // ------------------------------------------------------------------ waiter for the MMA issuer
-        int s = 0;
-        uint32_t ph = 0;
-        bool ok = true;                                      // lane 0's view; shared with warp 1 at every hand-over
-        for (int g = 0; g < ng1; ++g) {
-            if (lane == 0 && ok) ok = mbar_wait(smem_u32(&full1[s]), ph, ab);
-            if (++s == p.S1) { s = 0; ph ^= 1; }
-            __syncwarp();
-            pair_sync_or(lane == 0 && !ok);
-        }
-        s = 0;
         ph = 0;
         int i2 = 0;
-        for (int j = c; j < p.n_chunks; j += p.C, ++i2) {
-            for (int g = 0; g < ng2; ++g) {
-                if (lane == 0) {
-                    if (g == 0) {
-                        // every slice of T has landed in this block's buffer; the accumulator buffer is free again
-                        if (ok && i2 == 0) ok = mbar_wait_cluster(smem_u32(&tready_bar), 0, ab);
-                        if (ok) ok = mbar_wait(smem_u32(&out_empty[i2 & 1]), ((i2 >> 1) & 1) ^ 1, ab);
+        for (int j = c; j < p.n_chunks && ok; j += p.C, ++i2) {
+            const uint32_t d_tmem = tmem_base + (uint32_t)(i2 & 1) * 256u;
+            ok = mbar_wait_uniform(smem_u32(&out_empty[i2 & 1]), ((i2 >> 1) & 1) ^ 1, ab);   // accumulator buffer drained
+            for (int kb = 0; kb < p.kb2 && ok; ++kb) {
+                ok = mbar_wait_uniform(smem_u32(&full2[s]), ph, ab);
+                if (!ok) break;
+                if (i2 == 0 && kb < 8 && lane == 0) { LRD_TS(24 + kb); }
+                tc_fence_after();
+                const uint32_t q_src = ring2_base + s * p.stage2_bytes;
+                const uint64_t bd = a_desc0 + ((q_src >> 4) & 0x3FFFu);
+                const int nks = min(4, p.ks2 - kb * 4);
+                if (elect_one()) {
+                    for (int kk = 0; kk < nks; ++kk) {
+                        const uint32_t ks = (uint32_t)(kb * 4 + kk);      // 16-column step within T
+                        const uint64_t ad = t_desc0 + (((ks >> p.t_steps_lg) * t_atom_bytes + (ks & ((1u << p.t_steps_lg) - 1u)) * 32u) >> 4);
+                        mma_bf16_ss(d_tmem, ad, bd + 2u * kk, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
                     }
-                    if (ok) ok = mbar_wait(smem_u32(&full2[s]), ph, ab);
+                    mma_commit(smem_u32(&empty2[s]));
+                    if (kb == p.kb2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
                 }
-                if (++s == p.S2) { s = 0; ph ^= 1; }
                 __syncwarp();
-                pair_sync_or(lane == 0 && !ok);
+                if (i2 == 0 && kb < 8 && lane == 0) { LRD_TS(32 + kb); }
+                if (++s == p.S2) { s = 0; ph ^= 1; }
             }
         }
+        if (lane == 0) { LRD_TS(9); }
+        cluster_wait();        // barrier 1 (long complete: every peer has pushed into this block)
+        cluster_arrive();      // barrier 2: this block has received everything its peers send (T was complete above)
     } else {
         // ------------------------------------------------------------------ gather + epilogue
         const int q = warp % 4;                              // tensor-memory lanes [32 q, 32 q + 32)
         const int row = q * 32 + lane;                       // row of the 128-row tile
+        const int et = (warp - 2) * 32 + lane;               // index among the 128 epilogue threads
+        const bool lead_warp = (warp == 2);                  // issues this block's bulk copies and stores (elect.sync)
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         bool ok = mbar_wait_warp(smem_u32(&tacc_bar), 0, ab);   // warp-uniform from here on
         tc_fence_after();
+        if (lead_warp && lane == 0) { LRD_TS(10); }
         if (ok) {
             for (int piece = 0; piece * 16 < p.RS; ++piece) {
                 uint32_t v[16];
@@ -269,92 +265,114 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         // the four warps have written it, one thread copies it into every peer's buffer (bulk DSMEM copy that
         // completes on the peer's barrier) and, if asked, stores it to T_save.  The accumulator columns of
         // the slice are free for phase 2 from here on.
+        if (lead_warp && lane == 0) { LRD_TS(17); }
         fence_proxy_async_smem();
         tc_fence_before();
+        cluster_wait();        // barrier 1: the peers' barriers exist
         named_bar_sync(2, 128);
-        if (q == 0 && lane == 0 && ok) {
-            const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;
-            for (int t = 1; t < p.C; ++t) {
-                const uint32_t peer = (uint32_t)((c + t) % p.C);
-                dsmem_bulk_copy(slice, slice, 256u * (uint32_t)p.RS, smem_u32(&tready_bar), peer);
-            }
-            mbar_arrive(smem_u32(&tready_bar));
-            if (p.has_tsave) {
-                for (int a = 0; a * p.taw < p.RS; ++a)
-                    tma_store_2d(&tmT, slice + (uint32_t)a * t_atom_bytes, c * p.RS + a * p.taw, m0);
-                tma_store_commit();
-            }
-        }
-        __syncwarp();
-        // Epilogue: 32 columns at a time through a [32 rows x 64 B] slab of this warp (64-byte swizzle),
-        // two slabs in rotation; each slab leaves by its own TMA store.
-        const uint32_t slab_base = staging_base + q * 2 * kSlabBytes;
-        const uint32_t slab_row = (uint32_t)lane * 64u;
-        const uint32_t slab_xor = ((uint32_t)lane >> 1) & 3u;
-        int i = 0, sb = 0;
-        for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
-            const int buf = i & 1;
-            ok = mbar_wait_warp(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_tmem = lane_addr + (uint32_t)buf * 256u;
-            for (int g = 0; g * 32 < p.BN2; ++g, ++sb) {
-                const int colh = j * p.BN2 + g * 32;
-                if (colh >= p.N2) continue;                  // (uniform) nothing of this piece is inside Out
-                const uint32_t slab = slab_base + (sb & 1) * kSlabBytes;
-                // the 32 bias values of this piece: four 16-byte loads (same address in every lane), issued
-                // before the accumulator load so that both latencies overlap
-                uint4 bv[4] = {};
-                const bool bias_vec = p.bias && colh + 32 <= p.N2;
-                if (bias_vec) {
-                    const uint4* bp = reinterpret_cast<const uint4*>(p.bias + colh);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) bv[e] = __ldg(bp + e);
+        if (lead_warp) {
+            if (ok && elect_one()) {
+                LRD_TS(11);
+                const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;
+                for (int t = 1; t < p.C; ++t) {
+                    const uint32_t peer = (uint32_t)((c + t) % p.C);
+                    dsmem_bulk_copy(slice, slice, 256u * (uint32_t)p.RS, smem_u32(&tready_bar), peer);
                 }
-                uint32_t v[32];
-                tmem_ld_32x32(d_tmem + g * 32, v);
-                if (sb >= 2) {                               // the store that last read this slab has finished reading
-                    if (lane == 0) tma_store_wait_read<1>();
-                    __syncwarp();
-                }
-                tmem_ld_wait();
-                if (bias_vec) {
-                    const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        v[2 * e] = __float_as_uint(__uint_as_float(v[2 * e]) + __uint_as_float(bw[e] << 16));
-                        v[2 * e + 1] = __float_as_uint(__uint_as_float(v[2 * e + 1]) + __uint_as_float(bw[e] & 0xFFFF0000u));
-                    }
-                } else if (p.bias) {                         // ragged last piece
-                    for (int e = 0; e < 32; ++e)
-                        if (colh + e < p.N2) v[e] = __float_as_uint(__uint_as_float(v[e]) + __bfloat162float(p.bias[colh + e]));
-                }
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    st_shared_v4(slab + slab_row + (((uint32_t)cc ^ slab_xor) << 4),
-                                 pack_bf16(__uint_as_float(v[8 * cc]), __uint_as_float(v[8 * cc + 1])),
-                                 pack_bf16(__uint_as_float(v[8 * cc + 2]), __uint_as_float(v[8 * cc + 3])),
-                                 pack_bf16(__uint_as_float(v[8 * cc + 4]), __uint_as_float(v[8 * cc + 5])),
-                                 pack_bf16(__uint_as_float(v[8 * cc + 6]), __uint_as_float(v[8 * cc + 7])));
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_2d(&tmOut, slab, colh, m0 + q * 32);
+                mbar_arrive(smem_u32(&tready_bar));
+                if (p.has_tsave) {
+                    for (int a = 0; a * p.taw < p.RS; ++a)
+                        tma_store_2d(&tmT, slice + (uint32_t)a * t_atom_bytes, c * p.RS + a * p.taw, m0);
                     tma_store_commit();
                 }
+                LRD_TS(12);
+            }
+            __syncwarp();
+        }
+        // Epilogue: 64 columns at a time through a [128 rows x 128 B] slab (128-byte swizzle) that the four
+        // warps fill together, two slabs in rotation; each slab leaves by one TMA store.  The bias of a
+        // chunk is staged in shared memory while its MMAs run.
+        const uint32_t row_off = (uint32_t)row * 128u;
+        const uint32_t row_xor = (uint32_t)row & 7u;
+        int i = 0, sb = 0;
+        bool arrived2 = false;
+        for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
+            const int buf = i & 1;
+            if (p.bias) {                                    // bias_s[buf] was last read two chunks ago, before a barrier
+                for (int e = et; e < p.BN2; e += 128) {
+                    const int col = j * p.BN2 + e;
+                    bias_s[buf][e] = col < p.N2 ? __bfloat162float(p.bias[col]) : 0.f;
+                }
+            }
+            ok = mbar_wait_warp(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
+            ok = named_bar_and(3, 128, ok);                  // the four warps go on, or give up, together (and see the bias)
+            if (!ok) break;
+            if (!arrived2) { cluster_arrive(); arrived2 = true; }   // barrier 2 (T was complete before these MMAs)
+            if (lead_warp && lane == 0 && i == 0) { LRD_TS(13); }
+            tc_fence_after();
+            const uint32_t d_tmem = lane_addr + (uint32_t)buf * 256u;
+            for (int g = 0; g * 64 < p.BN2; ++g) {
+                const int col0 = j * p.BN2 + g * 64;
+                if (col0 >= p.N2) break;                     // (uniform) nothing of this piece is inside Out
+                const uint32_t slab = staging_base + (uint32_t)(sb & 1) * kSlabBytes;
+                if (sb >= 2) {                               // the store that last read this slab has finished reading
+                    if (lead_warp) tma_store_wait_read<1>();
+                    named_bar_sync(3, 128);
+                }
+                if (lead_warp && lane == 0 && sb < 4) { LRD_TS(40 + 4 * sb); }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(d_tmem + g * 64 + h * 32, v);
+                    tmem_ld_wait();
+                    if (p.bias) {
+                        const float4* bp = reinterpret_cast<const float4*>(&bias_s[buf][g * 64 + h * 32]);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float4 b4 = bp[e];
+                            v[4 * e] = __float_as_uint(__uint_as_float(v[4 * e]) + b4.x);
+                            v[4 * e + 1] = __float_as_uint(__uint_as_float(v[4 * e + 1]) + b4.y);
+                            v[4 * e + 2] = __float_as_uint(__uint_as_float(v[4 * e + 2]) + b4.z);
+                            v[4 * e + 3] = __float_as_uint(__uint_as_float(v[4 * e + 3]) + b4.w);
+                        }
+                    }
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc)
+                        st_shared_v4(slab + row_off + ((((uint32_t)(4 * h + cc)) ^ row_xor) << 4),
+                                     pack_bf16(__uint_as_float(v[8 * cc]), __uint_as_float(v[8 * cc + 1])),
+                                     pack_bf16(__uint_as_float(v[8 * cc + 2]), __uint_as_float(v[8 * cc + 3])),
+                                     pack_bf16(__uint_as_float(v[8 * cc + 4]), __uint_as_float(v[8 * cc + 5])),
+                                     pack_bf16(__uint_as_float(v[8 * cc + 6]), __uint_as_float(v[8 * cc + 7])));
+                }
+                if (lead_warp && lane == 0 && sb < 4) { LRD_TS(41 + 4 * sb); }
+                fence_proxy_async_smem();
+                named_bar_sync(2, 128);
+                if (lead_warp && lane == 0 && sb < 4) { LRD_TS(43 + 4 * sb); }
+                if (lead_warp) {
+                    if (elect_one()) {
+                        tma_store_2d(&tmOut, slab, col0, m0);
+                        tma_store_commit();
+                    }
+                    __syncwarp();
+                }
+                ++sb;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&out_empty[buf]));
         }
-        if (lane == 0) tma_store_wait_all<0>();
+        if (!arrived2) cluster_arrive();
+        if (lead_warp && lane == 0) { LRD_TS(14); }
+        if (lead_warp) tma_store_wait_read<0>();             // shared memory may go once the stores have read it
+        if (lead_warp && lane == 0) { LRD_TS(15); }
         __syncwarp();
     }
 
+    // Cluster barrier 2: no block leaves while a peer may still be reading its slice out of this block's
+    // shared memory (each block arrived once all slices addressed to it had landed).
+    cluster_wait();
     tc_fence_before();
     __syncthreads();
-    cluster_arrive();          // no block leaves while a peer may still write into its shared memory
-    cluster_wait();
+    if (threadIdx.x == 0) { LRD_TS(16); }
     if (warp == 1) {
         if (abort_flag) {
             for (int i = 0; i < 256; ++i) __nanosleep(1000);
@@ -365,15 +383,18 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
 }
 
 struct Plan {
-    int C, RS, swb, BN2, G1, S1, G2, S2;
+    int C, RS, swb, BN2, G1, S1, S2;
     uint32_t stage1_bytes, stage2_bytes, t_bytes, smem_bytes;
 };
+
+int g_tune_C = 0, g_tune_G1 = 0, g_tune_BN2 = 0;    // 0 = automatic
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // Column chunk width of phase 2: the block with the most chunks sets the pace, so minimise
 // (chunks of the busiest block) x width; wider chunks on ties (fewer, larger copies).
 int pick_bn2(int64_t N2, int C) {
+    if (g_tune_BN2) return g_tune_BN2;
     const int cands[3] = {256, 192, 128};
     int best = 128;
     int64_t best_cost = -1;
@@ -395,33 +416,32 @@ bool make_plan(const ChainArgs& a, Plan* out) {
     if (a.bias && !aligned16(a.bias)) return false;
     const int64_t tiles = (a.M + 127) / 128;
     const int t_bytes = (int)((a.r * 256 + 1023) / 1024 * 1024);      // 128 rows x r columns of bf16
-    const int kb1 = (int)((a.K1 + 63) / 64), kb2 = (int)((a.r + 63) / 64);
+    const int kb1 = (int)((a.K1 + 63) / 64);
     Plan best{};
     bool found = false;
     const int cands[3] = {4, 2, 1};
     for (int C : cands) {
+        if (g_tune_C && C != g_tune_C) continue;
         if (a.r % (16 * C)) continue;
         const int RS = (int)a.r / C;
         if (RS > 256) continue;
         const int swb = RS % 64 == 0 ? 128 : (RS % 32 == 0 ? 64 : 32);
         const int BN2 = pick_bn2(a.N2, C);
-        const int64_t ring = (int64_t)kSmemLimit - 1024 - t_bytes - (int64_t)kStagingBytes;
+        const int64_t ring1 = (int64_t)kSmemLimit - 1024 - t_bytes;
+        const int64_t ring2 = ring1 - (int64_t)kStagingBytes;
         const uint32_t kb1_bytes = kInTileBytes + 128u * RS, kb2_bytes = (uint32_t)BN2 * 128u;
-        // the most k-blocks per stage that still leave two stages (phase 1: a P box is at most 256 rows)
-        int G1 = 0, G2 = 0;
-        for (int g = 4; g >= 1; --g)
-            if (ring / ((int64_t)g * kb1_bytes) >= 2) { G1 = g; break; }
-        for (int g = 4; g >= 1; --g)
-            if (ring / ((int64_t)g * kb2_bytes) >= 2) { G2 = g; break; }
-        if (!G1 || !G2) continue;
+        if (ring2 < 2 * (int64_t)kb2_bytes) continue;
+        // phase 1: one k-block per stage (the finest pipeline) unless overridden
+        int G1 = g_tune_G1 ? g_tune_G1 : 1;
+        if (G1 > 4) G1 = 4;
         if (G1 > kb1) G1 = kb1;
-        if (G2 > kb2) G2 = kb2;
-        int S1 = (int)(ring / ((int64_t)G1 * kb1_bytes)), S2 = (int)(ring / ((int64_t)G2 * kb2_bytes));
+        if (ring1 < 2 * (int64_t)G1 * kb1_bytes) continue;
+        int S1 = (int)(ring1 / ((int64_t)G1 * kb1_bytes)), S2 = (int)(ring2 / (int64_t)kb2_bytes);
         if (S1 > kMaxStages) S1 = kMaxStages;
         if (S2 > kMaxStages) S2 = kMaxStages;
-        const uint32_t s1b = (uint32_t)G1 * kb1_bytes, s2b = (uint32_t)G2 * kb2_bytes;
-        const uint32_t used = (uint32_t)S1 * s1b > (uint32_t)S2 * s2b ? (uint32_t)S1 * s1b : (uint32_t)S2 * s2b;
-        Plan pl{C, RS, swb, BN2, G1, S1, G2, S2, s1b, s2b, (uint32_t)t_bytes, (uint32_t)(1024 + t_bytes + kStagingBytes + used)};
+        const uint32_t s1b = (uint32_t)G1 * kb1_bytes;
+        const uint32_t used1 = (uint32_t)S1 * s1b, used2 = kStagingBytes + (uint32_t)S2 * kb2_bytes;
+        Plan pl{C, RS, swb, BN2, G1, S1, S2, s1b, kb2_bytes, (uint32_t)t_bytes, 1024u + (uint32_t)t_bytes + (used1 > used2 ? used1 : used2)};
         // prefer the largest cluster whose blocks are all resident at once; else the smallest feasible
         if (!found) { best = pl; found = true; }
         if (tiles * C <= kNumSms) { best = pl; break; }
@@ -433,6 +453,12 @@ bool make_plan(const ChainArgs& a, Plan* out) {
 }
 
 }  // namespace
+
+void chain_tuning(int C, int G1, int BN2) {
+    g_tune_C = C;
+    g_tune_G1 = G1;
+    g_tune_BN2 = BN2;
+}
 
 bool chain_eligible(const ChainArgs& a) {
     Plan pl;
@@ -446,7 +472,7 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     bool ok = make_tmap_2d_bf16(&tIn, a.In, (uint64_t)a.M, (uint64_t)a.K1, (uint64_t)a.ld_in, 128, 64);
     ok = ok && make_tmap_2d_bf16(&tP, a.P, (uint64_t)a.K1, (uint64_t)a.r, (uint64_t)a.ldp, 64u * (uint32_t)pl.G1, (uint32_t)pl.swb / 2);
     ok = ok && make_tmap_2d_bf16(&tQ, a.Q, (uint64_t)a.N2, (uint64_t)a.r, (uint64_t)a.ldq, (uint32_t)pl.BN2, 64);
-    ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 32, 32);
+    ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 128, 64);
     if (a.T_save)
         ok = ok && make_tmap_2d_bf16(&tT, a.T_save, (uint64_t)a.M, (uint64_t)a.r, (uint64_t)a.ldt, 128, (uint32_t)pl.swb / 2);
     else
@@ -460,9 +486,10 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     p.ks2 = (int)a.r / 16;
     p.kb2 = (int)((a.r + 63) / 64);
     p.N2 = (int)a.N2;
-    p.G1 = pl.G1; p.S1 = pl.S1; p.G2 = pl.G2; p.S2 = pl.S2;
+    p.G1 = pl.G1; p.S1 = pl.S1; p.S2 = pl.S2;
     p.stage1_bytes = pl.stage1_bytes; p.stage2_bytes = pl.stage2_bytes; p.t_bytes = pl.t_bytes;
     p.taw = pl.swb / 2;
+    p.t_steps_lg = p.taw == 64 ? 2 : (p.taw == 32 ? 1 : 0);
     p.bias = (const __nv_bfloat16*)a.bias;
     p.has_tsave = a.T_save ? 1 : 0;
     p.timeout_flag = device_timeout_flag();

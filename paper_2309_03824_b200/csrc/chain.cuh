@@ -18,6 +18,9 @@ struct ChainArgs {
     lrd_dtype_t dtype;
 };
 
+// Overrides of the launch shape for benchmarking sweeps: cluster size, k-blocks per phase-1 stage,
+// phase-2 chunk width.  0 = automatic.  Not thread-safe against concurrent launches.
+void chain_tuning(int C, int G1, int BN2);
 bool chain_eligible(const ChainArgs& c);
 lrd_status_t chain_launch(const ChainArgs& c, cudaStream_t stream);
 

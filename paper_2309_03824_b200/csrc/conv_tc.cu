@@ -9,7 +9,7 @@
 //                       pixel chunks, fp32 partials added in a fixed order by filter_reduce_kernel)
 //
 // A tile is bh rows of one image (bh * W <= 128 pixels = the 128 MMA rows / the reduction chunk).
-// Warp roles as in the matrix-product kernel: TMA producer, MMA issuer, 4 epilogue warps, 1 waiter.
+// Warp roles as in the matrix-product kernel: TMA producer, MMA issuer (both issue under elect.sync from a converged warp), 4 epilogue warps.
 #include "common.cuh"
 #include "conv.cuh"
 #include "ptx.cuh"
@@ -21,7 +21,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 224;
+constexpr int kThreads = 192;
 constexpr int kStages = 4;
 constexpr uint32_t kTile = 128 * 128;               // one operand tile slot: 128 rows x 64 channels of bf16
 constexpr uint32_t kStageBytes = 3 * kTile;          // A slot + two 64-wide B slots (N = 128)
@@ -47,7 +47,7 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
     __shared__ int abort_flag;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
     const int n0 = blockIdx.x * 128, h0 = blockIdx.y * p.bh, img = blockIdx.z;
     const int nkc = (p.ka + 63) / 64;                  // 64-channel blocks per tap
     const int iters = 9 * nkc;
@@ -75,16 +75,17 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
     const uint32_t tmem_base = tmem_base_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 1;
-            for (int it = 0; it < iters; ++it) {
-                const int tap = it / nkc, cb = it % nkc;
-                const int kh = tap / 3, kw = tap % 3;
-                if (!mbar_wait(smem_u32(&empty_bar[s]), ph, ab)) break;
-                const uint32_t fb = smem_u32(&full_bar[s]);
+        // TMA producer: the whole warp runs the loop, one elected lane issues
+        int s = 0;
+        uint32_t ph = 1;
+        for (int it = 0; it < iters; ++it) {
+            const int tap = it / nkc, cb = it % nkc;
+            const int kh = tap / 3, kw = tap % 3;
+            if (!mbar_wait_uniform(smem_u32(&empty_bar[s]), ph, ab)) break;
+            const uint32_t fb = smem_u32(&full_bar[s]);
+            const uint32_t a_dst = smem_base + s * kStageBytes, b_dst = a_dst + kTile;
+            if (elect_one()) {
                 mbar_expect_tx(fb, stage_tx);
-                const uint32_t a_dst = smem_base + s * kStageBytes, b_dst = a_dst + kTile;
                 // image window of this tap: rows h0 + sign (kh - 1) ..., columns sign (kw - 1) ...; outside = zeros
                 tma_load_4d(a_dst, &tmImg, fb, cb * 64, p.sign * (kw - 1), h0 + p.sign * (kh - 1), img);
                 if (DGRAD) {           // B[n = i][k = o] = G[o][tap][i]: MN-major, rows o of this block, 64 columns of i per box
@@ -93,19 +94,22 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
                 } else {               // B[n = o][k = i] = G[o][tap][i]: K-major, 128 rows of o
                     tma_load_2d(b_dst, &tmG, fb, tap * p.g_ci + cb * 64, n0);
                 }
-                if (++s == kStages) { s = 0; ph ^= 1; }
             }
+            __syncwarp();
+            if (++s == kStages) { s = 0; ph ^= 1; }
         }
-        __syncwarp();
     } else if (warp == 1) {
+        // MMA issuer: converged warp, elect.sync around the issue
         constexpr uint32_t idesc = idesc_bf16(128, false, DGRAD);
         int s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (int it = 0; it < iters; ++it) {
-            ok = !pair_sync_or(false) && ok;
-            if (lane == 0 && ok) {
-                tc_fence_after();
-                const uint32_t a_src = smem_base + s * kStageBytes, b_src = a_src + kTile;
+            ok = mbar_wait_uniform(smem_u32(&full_bar[s]), ph, ab);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_src = smem_base + s * kStageBytes, b_src = a_src + kTile;
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
                     const uint64_t ad = smem_desc_sw128(a_src + kk * 32, 0, 1024);
@@ -115,20 +119,11 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
                 }
                 mma_commit(smem_u32(&empty_bar[s]));
             }
-            if (++s == kStages) s = 0;
-        }
-        if (lane == 0 && ok) mma_commit(smem_u32(&acc_bar));
-        __syncwarp();
-    } else if (warp == 6) {
-        int s = 0;
-        uint32_t ph = 0;
-        bool ok = true;
-        for (int it = 0; it < iters; ++it) {
-            if (lane == 0 && ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
-            if (++s == kStages) { s = 0; ph ^= 1; }
             __syncwarp();
-            pair_sync_or(lane == 0 && !ok);
+            if (++s == kStages) { s = 0; ph ^= 1; }
         }
+        if (ok && elect_one()) mma_commit(smem_u32(&acc_bar));
+        __syncwarp();
     } else {
         const int q = warp % 4;
         const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
@@ -192,7 +187,7 @@ filter_kernel(const __grid_constant__ CUtensorMap tmDout, const __grid_constant_
     __shared__ int abort_flag;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
     const int tap = blockIdx.x, kh = tap / 3, kw = tap % 3;
     const int m0 = (blockIdx.y / p.tiles_i) * 128, n0 = (blockIdx.y % p.tiles_i) * 128;
     const int c_begin = blockIdx.z * p.chunks_per_split;
@@ -227,32 +222,34 @@ filter_kernel(const __grid_constant__ CUtensorMap tmDout, const __grid_constant_
     const uint32_t tmem_base = tmem_base_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 1;
-            for (int ch = c_begin; ch < c_end; ++ch) {
-                const int img = ch / p.tiles_per_img, h0 = (ch % p.tiles_per_img) * p.bh;
-                if (!mbar_wait(smem_u32(&empty_bar[s]), ph, ab)) break;
-                const uint32_t fb = smem_u32(&full_bar[s]);
+        int s = 0;
+        uint32_t ph = 1;
+        for (int ch = c_begin; ch < c_end; ++ch) {
+            const int img = ch / p.tiles_per_img, h0 = (ch % p.tiles_per_img) * p.bh;
+            if (!mbar_wait_uniform(smem_u32(&empty_bar[s]), ph, ab)) break;
+            const uint32_t fb = smem_u32(&full_bar[s]);
+            const uint32_t dst = smem_base + s * kFStageBytes;
+            if (elect_one()) {
                 mbar_expect_tx(fb, 4u * box_bytes);
-                const uint32_t dst = smem_base + s * kFStageBytes;
                 tma_load_4d(dst, &tmDout, fb, m0, 0, h0, img);
                 tma_load_4d(dst + kTile, &tmDout, fb, m0 + 64, 0, h0, img);
                 tma_load_4d(dst + 2 * kTile, &tmIn, fb, n0, kw - 1, h0 + kh - 1, img);
                 tma_load_4d(dst + 3 * kTile, &tmIn, fb, n0 + 64, kw - 1, h0 + kh - 1, img);
-                if (++s == kFStages) { s = 0; ph ^= 1; }
             }
+            __syncwarp();
+            if (++s == kFStages) { s = 0; ph ^= 1; }
         }
-        __syncwarp();
     } else if (warp == 1) {
         constexpr uint32_t idesc = idesc_bf16(128, true, true);
         int s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (int ch = c_begin; ch < c_end; ++ch) {
-            ok = !pair_sync_or(false) && ok;
-            if (lane == 0 && ok) {
-                tc_fence_after();
-                const uint32_t a_src = smem_base + s * kFStageBytes, b_src = a_src + 2 * kTile;
+            ok = mbar_wait_uniform(smem_u32(&full_bar[s]), ph, ab);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_src = smem_base + s * kFStageBytes, b_src = a_src + 2 * kTile;
+            if (elect_one()) {
                 for (int kk = 0; kk < ksteps; ++kk) {
                     const uint64_t ad = smem_desc_sw128(a_src + kk * 2048, kTile, 1024);
                     const uint64_t bd = smem_desc_sw128(b_src + kk * 2048, kTile, 1024);
@@ -260,20 +257,11 @@ filter_kernel(const __grid_constant__ CUtensorMap tmDout, const __grid_constant_
                 }
                 mma_commit(smem_u32(&empty_bar[s]));
             }
-            if (++s == kFStages) s = 0;
-        }
-        if (lane == 0 && ok) mma_commit(smem_u32(&acc_bar));
-        __syncwarp();
-    } else if (warp == 6) {
-        int s = 0;
-        uint32_t ph = 0;
-        bool ok = true;
-        for (int ch = c_begin; ch < c_end; ++ch) {
-            if (lane == 0 && ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
-            if (++s == kFStages) { s = 0; ph ^= 1; }
             __syncwarp();
-            pair_sync_or(lane == 0 && !ok);
+            if (++s == kFStages) { s = 0; ph ^= 1; }
         }
+        if (ok && elect_one()) mma_commit(smem_u32(&acc_bar));
+        __syncwarp();
     } else {
         const int q = warp % 4;
         const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);

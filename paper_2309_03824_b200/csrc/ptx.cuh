@@ -41,7 +41,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait.  Returns false when the barrier did not flip within the limit or another
 // thread of the block has already given up; the caller then leaves its loop and the block
 // tears down in order.
-constexpr uint32_t kWaitSpinFast = 2048;
+constexpr uint32_t kWaitSpinFast = 1u << 14;
 constexpr uint32_t kWaitSpinLimit = 1u << 22;
 struct AbortCtx {
     volatile int* flag;        // shared memory: set by the first thread of the block that gives up
@@ -50,12 +50,21 @@ struct AbortCtx {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const AbortCtx& ab) {
     for (uint32_t it = 0; it < kWaitSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(it < kWaitSpinFast ? 20 : 128);      // a failed try backs off: hot polling starves the issuing warps
-        if (it >= kWaitSpinFast && *ab.flag) return false;
+        if (it >= kWaitSpinFast) {                       // a try suspends in hardware for a while by itself; back
+            __nanosleep(64);                             // off only when the wait is clearly a long one
+            if (*ab.flag) return false;
+        }
     }
     *ab.flag = 1;
     if (ab.global_flag) atomicExch(ab.global_flag, 1u);
     return false;
+}
+
+// The same wait executed by a whole converged warp, with a warp-uniform result (the warp stays
+// converged, so that an elect.sync region can follow).
+__device__ __forceinline__ bool mbar_wait_uniform(uint32_t bar, uint32_t parity, const AbortCtx& ab) {
+    const bool ok = mbar_wait(bar, parity, ab);
+    return __all_sync(0xffffffffu, ok) != 0;
 }
 
 // Warp-wide wait for the long waits of the epilogue warps: lane 0 polls with a sleep between tries
@@ -67,8 +76,10 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, co
         ok = false;
         for (uint32_t it = 0; it < kWaitSpinLimit; ++it) {
             if (mbar_try_wait(bar, parity)) { ok = true; break; }
-            __nanosleep(it < 64 ? 32 : 256);
-            if (it >= 64 && *ab.flag) break;
+            if (it >= 256) {
+                __nanosleep(64);
+                if (*ab.flag) break;
+            }
         }
         if (!ok && !*ab.flag) {
             *ab.flag = 1;
@@ -108,6 +119,11 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     *ab.flag = 1;
     if (ab.global_flag) atomicExch(ab.global_flag, 1u);
     return false;
+}
+
+__device__ __forceinline__ bool mbar_wait_cluster_uniform(uint32_t bar, uint32_t parity, const AbortCtx& ab) {
+    const bool ok = mbar_wait_cluster(bar, parity, ab);
+    return __all_sync(0xffffffffu, ok) != 0;
 }
 
 // ---- proxies and fences ---------------------------------------------------------------------
@@ -190,18 +206,6 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Rendezvous of two warps on named barrier 1 that also ORs a flag across them (no shared-memory
-// access: the MMA-issuing thread must not read shared memory between a tcgen05.commit and its
-// next MMAs, because such a read waits for the committed MMAs to finish and drains the pipe).
-// Every lane of both warps calls it, convergently.
-__device__ __forceinline__ bool pair_sync_or(bool flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 64, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r) : "r"(flag ? 1u : 0u) : "memory");
-    return r != 0;
-}
-
 // ---- descriptors ------------------------------------------------------------------------------
 // Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
 //   K-major operand  (rows of 64 bf16 = 128 B, 8-row groups of 1024 B): lbo unused, sbo = 1024.
@@ -263,6 +267,14 @@ __device__ __forceinline__ void dsmem_bulk_copy(uint32_t dst_local_addr, uint32_
 }
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// Barrier over `nthreads` threads that also ANDs a predicate across them.
+__device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tbar.red.and.pred p, %1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"(id), "r"(nthreads), "r"(pred ? 1u : 0u) : "memory");
+    return r != 0;
 }
 __device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");

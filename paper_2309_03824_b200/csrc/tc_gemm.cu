@@ -7,7 +7,7 @@
 //
 // One 128 x BN output tile per block.  Warp 0 issues TMA loads, warp 1 owns tensor memory and
 // issues the MMAs, warps 2-5 read the accumulator (each its own quarter of the 128 lanes) and
-// store, warp 6 waits on the stage barriers for warp 1.  Both operands may be K-major (reduction index contiguous) or MN-major (row / column
+// store.  The single-thread instructions are issued under elect.sync by a converged warp.  Both operands may be K-major (reduction index contiguous) or MN-major (row / column
 // index contiguous), which covers every product of the forward and backward pass without a
 // transposed copy.
 #include "common.cuh"
@@ -21,7 +21,7 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 224;
+constexpr int kThreads = 192;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
 
 // ONES: every stage carries one more 64-wide MN-major block of B that holds 1.0 everywhere and is never
@@ -62,7 +62,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int kb_begin = blockIdx.z * p.kb_per_split;
     const int kb_end = min(kb_begin + p.kb_per_split, p.kb_total);
@@ -94,17 +94,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tmem_base = tmem_base_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            int it = 0;
-            for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
-                if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, ab)) break;
-                const uint32_t fb = smem_u32(&full_bar[s]);
+        // TMA producer: the whole warp runs the loop, one elected lane issues (operands stay uniform)
+        int it = 0;
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1;
+            if (!mbar_wait_uniform(smem_u32(&empty_bar[s]), ph ^ 1, ab)) break;
+            const uint32_t fb = smem_u32(&full_bar[s]);
+            const uint32_t a_dst = smem_base + s * C::STAGE_BYTES;
+            const uint32_t b_dst = a_dst + A_STAGE_BYTES;
+            const int k0 = kb * BK;
+            if (elect_one()) {
                 mbar_expect_tx(fb, A_STAGE_BYTES + BN * BK * 2);
-                const uint32_t a_dst = smem_base + s * C::STAGE_BYTES;
-                const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                const int k0 = kb * BK;
                 if (A_MN) {
 #pragma unroll
                     for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * 8192, &tmA, fb, m0 + 64 * j, k0);
@@ -118,20 +119,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tma_load_2d(b_dst, &tmB, fb, k0, n0);
                 }
             }
+            __syncwarp();
         }
-        __syncwarp();
     } else if (warp == 1) {
-        // MMA issuer.  It never waits on a barrier itself (a shared-memory read behind a tcgen05.commit
-        // stalls until the committed MMAs finish): warp 6 waits and hands each ready stage over.
+        // MMA issuer: converged warp, elect.sync around the issue
         const uint32_t idesc = idesc_bf16(BN + ((ONES && blockIdx.x == 0) ? 16 : 0), A_MN, B_MN);
         int s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (int kb = kb_begin; kb < kb_end; ++kb) {
-            ok = !pair_sync_or(false) && ok;
-            if (lane == 0 && ok) {
-                tc_fence_after();
-                const uint32_t a_src = smem_base + s * C::STAGE_BYTES;
-                const uint32_t b_src = a_src + A_STAGE_BYTES;
+            ok = mbar_wait_uniform(smem_u32(&full_bar[s]), ph, ab);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_src = smem_base + s * C::STAGE_BYTES;
+            const uint32_t b_src = a_src + A_STAGE_BYTES;
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; ++kk) {
                     const uint64_t ad = A_MN ? smem_desc_sw128(a_src + kk * 2048, 8192, 1024)
@@ -142,20 +144,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 mma_commit(smem_u32(&empty_bar[s]));
             }
-            if (++s == STAGES) s = 0;
-        }
-        if (lane == 0 && ok) mma_commit(smem_u32(&acc_bar));
-        __syncwarp();
-    } else if (warp == 6) {
-        int s = 0;
-        uint32_t ph = 0;
-        bool ok = true;
-        for (int kb = kb_begin; kb < kb_end; ++kb) {
-            if (lane == 0 && ok) ok = mbar_wait(smem_u32(&full_bar[s]), ph, ab);
-            if (++s == STAGES) { s = 0; ph ^= 1; }
             __syncwarp();
-            pair_sync_or(lane == 0 && !ok);
+            if (++s == STAGES) { s = 0; ph ^= 1; }
         }
+        if (ok && elect_one()) mma_commit(smem_u32(&acc_bar));
+        __syncwarp();
     } else {
         const int quarter = warp % 4;                      // lanes [32 q, 32 q + 32) of tensor memory
         const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);

@@ -114,6 +114,10 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     cluster_arrive();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // Everything above touched only this block's own shared and tensor memory, so it may overlap the tail
+    // of the previous kernel in the stream; global memory is first read (and written) below this line.
+    griddep_launch_dependents();
+    griddep_wait();
     if (threadIdx.x == 0) { LRD_TS(1); }
 
     if (warp == 0) {
@@ -161,7 +165,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         }
         if (lane == 0) { LRD_TS(5); }
         cluster_wait();        // barrier 1
-        cluster_arrive();      // barrier 2
+        cluster_arrive_relaxed();   // barrier 2 (progress only)
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         int s = 0;
@@ -233,7 +237,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         }
         if (lane == 0) { LRD_TS(9); }
         cluster_wait();        // barrier 1 (long complete: every peer has pushed into this block)
-        cluster_arrive();      // barrier 2: this block has received everything its peers send (T was complete above)
+        cluster_arrive_relaxed();   // barrier 2: this block has received everything its peers send (T was complete above)
     } else {
         // ------------------------------------------------------------------ gather + epilogue
         const int q = warp % 4;                              // tensor-memory lanes [32 q, 32 q + 32)
@@ -306,7 +310,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             ok = mbar_wait_warp(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
             ok = named_bar_and(3, 128, ok);                  // the four warps go on, or give up, together (and see the bias)
             if (!ok) break;
-            if (!arrived2) { cluster_arrive(); arrived2 = true; }   // barrier 2 (T was complete before these MMAs)
+            if (!arrived2) { cluster_arrive_relaxed(); arrived2 = true; }   // barrier 2 (T was complete before these MMAs)
             if (lead_warp && lane == 0 && i == 0) { LRD_TS(13); }
             tc_fence_after();
             const uint32_t d_tmem = lane_addr + (uint32_t)buf * 256u;
@@ -360,7 +364,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&out_empty[buf]));
         }
-        if (!arrived2) cluster_arrive();
+        if (!arrived2) cluster_arrive_relaxed();
         if (lead_warp && lane == 0) { LRD_TS(14); }
         if (lead_warp) tma_store_wait_read<0>();             // shared memory may go once the stores have read it
         if (lead_warp && lane == 0) { LRD_TS(15); }
@@ -406,6 +410,33 @@ int pick_bn2(int64_t N2, int C) {
     return best;
 }
 
+// Clusters of C blocks that can be resident at once (a cluster needs C free SMs inside one GPC).
+int max_active_clusters(int C) {
+    static int cache[5] = {0, 0, 0, 0, 0};
+    if (C < 2 || C > 4) return kNumSms;
+    if (cache[C] == 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)C, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = kSmemLimit;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)C;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, chain_kernel, &cfg) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            n = (kNumSms - 20) / C;                     // no answer (no device yet): a cautious guess
+        }
+        cache[C] = n;
+    }
+    return cache[C];
+}
+
 bool make_plan(const ChainArgs& a, Plan* out) {
     if (a.dtype != LRD_BF16 || a.M < 1 || a.K1 < 1 || a.N2 < 1) return false;
     if (a.r < 16 || a.r > 512 || a.r % 16) return false;
@@ -444,7 +475,7 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         Plan pl{C, RS, swb, BN2, G1, S1, S2, s1b, kb2_bytes, (uint32_t)t_bytes, 1024u + (uint32_t)t_bytes + (used1 > used2 ? used1 : used2)};
         // prefer the largest cluster whose blocks are all resident at once; else the smallest feasible
         if (!found) { best = pl; found = true; }
-        if (tiles * C <= kNumSms) { best = pl; break; }
+        if (tiles <= max_active_clusters(C)) { best = pl; break; }
         best = pl;
     }
     if (!found) return false;
@@ -505,13 +536,15 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = pl.smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)pl.C;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // the kernel waits (griddepcontrol.wait) before it touches global memory
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, chain_kernel, tIn, tP, tQ, tOut, tT, p) != cudaSuccess) return LRD_ERR_CUDA;
     count_launch();
     return LRD_OK;

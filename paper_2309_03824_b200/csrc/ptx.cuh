@@ -236,6 +236,14 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n, bool a_mn_major, bool b
            ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start while its predecessor in
+// the stream is still running.  launch_dependents: this block no longer holds the next kernel back.
+// wait: returns once the predecessor has completed and its memory operations are visible; nothing
+// before it may touch global memory.  Both are no-ops in a kernel launched without the attribute.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- clusters -------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -243,6 +251,9 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
     return r;
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// Arrival without release semantics: signals progress only (a release waits for this block's
+// outstanding asynchronous copies, which can take microseconds right after a push).
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cluster_nctarank() {
     uint32_t r;

@@ -116,7 +116,7 @@ lrd_status_t lrd_set_path(lrd_path_t path);
 
 /* Launch-shape overrides of the fused chain kernel, for measurement sweeps (no counterpart in the
  * paper): blocks per cluster (1, 2 or 4), 64-deep k-blocks per pipeline stage of the first product
- * (1..4), column-chunk width of the second product (128, 192 or 256).  0 = automatic (the default).
+ * (1..4), column-chunk width of the second product (64, 128, 192 or 256).  0 = automatic (the default).
  * A shape the override makes infeasible falls back to the unfused products.  Process-wide, not
  * thread-safe against concurrent launches.  Returns LRD_ERR_INVALID_ARG for values outside the lists. */
 lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chunk_columns);

@@ -36,8 +36,8 @@ constexpr int kThreads = 192;
 constexpr int kMaxStages = 12;
 constexpr uint32_t kSmemLimit = 224 * 1024;         // dynamic shared memory; the rest is left for the barriers and the bias
 constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile of one k-block: 128 rows x 64 k
-constexpr uint32_t kSlabBytes = 128 * 64 * 2;       // epilogue slab: 128 rows x 64 columns of bf16
-constexpr uint32_t kStagingBytes = 2 * kSlabBytes;
+constexpr uint32_t kSlabBytes = 32 * 32 * 2;        // epilogue slab of one warp: 32 rows x 32 columns of bf16
+constexpr uint32_t kStagingBytes = 4 * 2 * kSlabBytes;
 
 struct ChainParams {
     int C, RS, swb, BN2, n_chunks, kb1, ks2, kb2, N2;
@@ -80,6 +80,14 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     // phase-1 stage: G1 In tiles, then the P boxes (one per column atom, 64 G1 rows tall)
     const uint32_t p_box_bytes = 64u * (uint32_t)p.G1 * (uint32_t)p.swb;
 
+    if (warp == 0 && lane >= 1 && lane <= kMaxStages) {      // the stage barriers, one stage per lane
+        const int s = lane - 1;
+        mbar_init(smem_u32(&full1[s]), 1);
+        mbar_init(smem_u32(&empty1[s]), 1);
+        mbar_init(smem_u32(&full2[s]), 1);
+        mbar_init(smem_u32(&empty2[s]), 1);
+        fence_mbar_init();
+    }
     if (threadIdx.x == 0) {
         LRD_TS(0);
         abort_flag = 0;
@@ -87,12 +95,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         prefetch_tmap(&tmP);
         prefetch_tmap(&tmQ);
         prefetch_tmap(&tmOut);
-        for (int s = 0; s < kMaxStages; ++s) {
-            mbar_init(smem_u32(&full1[s]), 1);
-            mbar_init(smem_u32(&empty1[s]), 1);
-            mbar_init(smem_u32(&full2[s]), 1);
-            mbar_init(smem_u32(&empty2[s]), 1);
-        }
         mbar_init(smem_u32(&tacc_bar), 1);
         // T complete = this block's own slice written (one arrival) + the peers' slices landed (bytes)
         mbar_init(smem_u32(&tready_bar), 2);
@@ -245,24 +247,31 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         const int et = (warp - 2) * 32 + lane;               // index among the 128 epilogue threads
         const bool lead_warp = (warp == 2);                  // issues this block's bulk copies and stores (elect.sync)
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        bool ok = mbar_wait_warp(smem_u32(&tacc_bar), 0, ab);   // warp-uniform from here on
+        bool ok = mbar_wait_uniform(smem_u32(&tacc_bar), 0, ab);   // warp-uniform from here on
         tc_fence_after();
         if (lead_warp && lane == 0) { LRD_TS(10); }
         if (ok) {
-            for (int piece = 0; piece * 16 < p.RS; ++piece) {
-                uint32_t v[16];
-                tmem_ld_32x16(lane_addr + piece * 16, v);
+            // 32 columns per step (two tensor-memory loads in flight, one wait), a 16-column tail if RS / 16 is odd
+            for (int col = 0; col < p.RS; col += 32) {
+                uint32_t v[32];
+                const bool two = col + 32 <= p.RS;
+                tmem_ld_32x16(lane_addr + col, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                if (two) tmem_ld_32x16(lane_addr + col + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
                 tmem_ld_wait();
-                uint32_t w[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-                const int gc = c * p.RS + piece * 16;        // first column of this piece within T
-                const uint32_t row_addr = t_base + (uint32_t)(gc / p.taw) * t_atom_bytes + (uint32_t)row * t_sw;
-                const uint32_t chunk0 = (uint32_t)(gc % p.taw) / 8u;
-                const uint32_t sw_xor = (((uint32_t)row * t_sw) >> 7) & (t_sw / 16u - 1u);
+                for (int half = 0; half < 2; ++half) {
+                    if (half == 1 && !two) break;
+                    uint32_t w[8];
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    st_shared_v4(row_addr + (((chunk0 + h) ^ sw_xor) << 4), w[4 * h], w[4 * h + 1], w[4 * h + 2], w[4 * h + 3]);
+                    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(v[16 * half + 2 * e]), __uint_as_float(v[16 * half + 2 * e + 1]));
+                    const int gc = c * p.RS + col + 16 * half;   // first column of this piece within T
+                    const uint32_t row_addr = t_base + (uint32_t)(gc / p.taw) * t_atom_bytes + (uint32_t)row * t_sw;
+                    const uint32_t chunk0 = (uint32_t)(gc % p.taw) / 8u;
+                    const uint32_t sw_xor = (((uint32_t)row * t_sw) >> 7) & (t_sw / 16u - 1u);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        st_shared_v4(row_addr + (((chunk0 + h) ^ sw_xor) << 4), w[4 * h], w[4 * h + 1], w[4 * h + 2], w[4 * h + 3]);
+                }
             }
         }
         // The slice [c RS, (c+1) RS) is whole atoms, i.e. one contiguous range of this block's T buffer: after
@@ -292,11 +301,12 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             }
             __syncwarp();
         }
-        // Epilogue: 64 columns at a time through a [128 rows x 128 B] slab (128-byte swizzle) that the four
-        // warps fill together, two slabs in rotation; each slab leaves by one TMA store.  The bias of a
-        // chunk is staged in shared memory while its MMAs run.
-        const uint32_t row_off = (uint32_t)row * 128u;
-        const uint32_t row_xor = (uint32_t)row & 7u;
+        // Epilogue: each warp on its own.  32 columns of its 32 rows at a time go through a [32 rows x 64 B]
+        // slab of the warp (64-byte swizzle, two slabs in rotation) and leave by one TMA store each.  The bias
+        // of a chunk is staged in shared memory while its MMAs run.
+        const uint32_t slab0 = staging_base + (uint32_t)(warp - 2) * 2u * kSlabBytes;
+        const uint32_t row_off = (uint32_t)lane * 64u;
+        const uint32_t row_xor = ((uint32_t)lane >> 1) & 3u;
         int i = 0, sb = 0;
         bool arrived2 = false;
         for (int j = c; j < p.n_chunks && ok; j += p.C, ++i) {
@@ -307,7 +317,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                     bias_s[buf][e] = col < p.N2 ? __bfloat162float(p.bias[col]) : 0.f;
                 }
             }
-            ok = mbar_wait_warp(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
+            ok = mbar_wait_uniform(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
             ok = named_bar_and(3, 128, ok);                  // the four warps go on, or give up, together (and see the bias)
             if (!ok) break;
             if (!arrived2) { cluster_arrive_relaxed(); arrived2 = true; }   // barrier 2 (T was complete before these MMAs)
@@ -317,48 +327,46 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             for (int g = 0; g * 64 < p.BN2; ++g) {
                 const int col0 = j * p.BN2 + g * 64;
                 if (col0 >= p.N2) break;                     // (uniform) nothing of this piece is inside Out
-                const uint32_t slab = staging_base + (uint32_t)(sb & 1) * kSlabBytes;
-                if (sb >= 2) {                               // the store that last read this slab has finished reading
-                    if (lead_warp) tma_store_wait_read<1>();
-                    named_bar_sync(3, 128);
-                }
-                if (lead_warp && lane == 0 && sb < 4) { LRD_TS(40 + 4 * sb); }
+                uint32_t v[64];                              // both halves are loaded before the first is converted
+                tmem_ld_32x32(d_tmem + g * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                tmem_ld_32x32(d_tmem + g * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+                if (lead_warp && lane == 0 && sb < 8) { LRD_TS(40 + 2 * sb); }
+                tmem_ld_wait();
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t v[32];
-                    tmem_ld_32x32(d_tmem + g * 64 + h * 32, v);
-                    tmem_ld_wait();
+                for (int h = 0; h < 2; ++h, ++sb) {
+                    if (col0 + 32 * h >= p.N2) break;        // (uniform)
+                    const uint32_t slab = slab0 + (uint32_t)(sb & 1) * kSlabBytes;
+                    if (sb >= 2) {                           // the store that last read this slab has finished reading
+                        tma_store_wait_read<1>();            // (only the lane that issued the stores has any to wait for)
+                        __syncwarp();
+                    }
                     if (p.bias) {
                         const float4* bp = reinterpret_cast<const float4*>(&bias_s[buf][g * 64 + h * 32]);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
                             const float4 b4 = bp[e];
-                            v[4 * e] = __float_as_uint(__uint_as_float(v[4 * e]) + b4.x);
-                            v[4 * e + 1] = __float_as_uint(__uint_as_float(v[4 * e + 1]) + b4.y);
-                            v[4 * e + 2] = __float_as_uint(__uint_as_float(v[4 * e + 2]) + b4.z);
-                            v[4 * e + 3] = __float_as_uint(__uint_as_float(v[4 * e + 3]) + b4.w);
+                            v[32 * h + 4 * e] = __float_as_uint(__uint_as_float(v[32 * h + 4 * e]) + b4.x);
+                            v[32 * h + 4 * e + 1] = __float_as_uint(__uint_as_float(v[32 * h + 4 * e + 1]) + b4.y);
+                            v[32 * h + 4 * e + 2] = __float_as_uint(__uint_as_float(v[32 * h + 4 * e + 2]) + b4.z);
+                            v[32 * h + 4 * e + 3] = __float_as_uint(__uint_as_float(v[32 * h + 4 * e + 3]) + b4.w);
                         }
                     }
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc)
-                        st_shared_v4(slab + row_off + ((((uint32_t)(4 * h + cc)) ^ row_xor) << 4),
-                                     pack_bf16(__uint_as_float(v[8 * cc]), __uint_as_float(v[8 * cc + 1])),
-                                     pack_bf16(__uint_as_float(v[8 * cc + 2]), __uint_as_float(v[8 * cc + 3])),
-                                     pack_bf16(__uint_as_float(v[8 * cc + 4]), __uint_as_float(v[8 * cc + 5])),
-                                     pack_bf16(__uint_as_float(v[8 * cc + 6]), __uint_as_float(v[8 * cc + 7])));
-                }
-                if (lead_warp && lane == 0 && sb < 4) { LRD_TS(41 + 4 * sb); }
-                fence_proxy_async_smem();
-                named_bar_sync(2, 128);
-                if (lead_warp && lane == 0 && sb < 4) { LRD_TS(43 + 4 * sb); }
-                if (lead_warp) {
+                        st_shared_v4(slab + row_off + ((((uint32_t)cc) ^ row_xor) << 4),
+                                     pack_bf16(__uint_as_float(v[32 * h + 8 * cc]), __uint_as_float(v[32 * h + 8 * cc + 1])),
+                                     pack_bf16(__uint_as_float(v[32 * h + 8 * cc + 2]), __uint_as_float(v[32 * h + 8 * cc + 3])),
+                                     pack_bf16(__uint_as_float(v[32 * h + 8 * cc + 4]), __uint_as_float(v[32 * h + 8 * cc + 5])),
+                                     pack_bf16(__uint_as_float(v[32 * h + 8 * cc + 6]), __uint_as_float(v[32 * h + 8 * cc + 7])));
+                    fence_proxy_async_smem();
+                    __syncwarp();
                     if (elect_one()) {
-                        tma_store_2d(&tmOut, slab, col0, m0);
+                        tma_store_2d(&tmOut, slab, col0 + 32 * h, m0 + q * 32);
                         tma_store_commit();
                     }
                     __syncwarp();
                 }
-                ++sb;
+                if (lead_warp && lane == 0 && sb <= 8) { LRD_TS(41 + 2 * (sb - 2)); }
             }
             tc_fence_before();
             __syncwarp();
@@ -366,7 +374,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         }
         if (!arrived2) cluster_arrive_relaxed();
         if (lead_warp && lane == 0) { LRD_TS(14); }
-        if (lead_warp) tma_store_wait_read<0>();             // shared memory may go once the stores have read it
+        tma_store_wait_read<0>();                            // shared memory may go once the stores have read it
         if (lead_warp && lane == 0) { LRD_TS(15); }
         __syncwarp();
     }
@@ -462,8 +470,9 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         const int64_t ring2 = ring1 - (int64_t)kStagingBytes;
         const uint32_t kb1_bytes = kInTileBytes + 128u * RS, kb2_bytes = (uint32_t)BN2 * 128u;
         if (ring2 < 2 * (int64_t)kb2_bytes) continue;
-        // phase 1: one k-block per stage (the finest pipeline) unless overridden
-        int G1 = g_tune_G1 ? g_tune_G1 : 1;
+        // phase 1: one k-block per stage (the finest pipeline); two for a short reduction, where the number of
+        // copies counts for more than the depth of the ring
+        int G1 = g_tune_G1 ? g_tune_G1 : (kb1 <= 16 ? 2 : 1);
         if (G1 > 4) G1 = 4;
         if (G1 > kb1) G1 = kb1;
         if (ring1 < 2 * (int64_t)G1 * kb1_bytes) continue;
@@ -503,7 +512,7 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     bool ok = make_tmap_2d_bf16(&tIn, a.In, (uint64_t)a.M, (uint64_t)a.K1, (uint64_t)a.ld_in, 128, 64);
     ok = ok && make_tmap_2d_bf16(&tP, a.P, (uint64_t)a.K1, (uint64_t)a.r, (uint64_t)a.ldp, 64u * (uint32_t)pl.G1, (uint32_t)pl.swb / 2);
     ok = ok && make_tmap_2d_bf16(&tQ, a.Q, (uint64_t)a.N2, (uint64_t)a.r, (uint64_t)a.ldq, (uint32_t)pl.BN2, 64);
-    ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 128, 64);
+    ok = ok && make_tmap_2d_bf16(&tOut, a.Out, (uint64_t)a.M, (uint64_t)a.N2, (uint64_t)a.ld_out, 32, 32);
     if (a.T_save)
         ok = ok && make_tmap_2d_bf16(&tT, a.T_save, (uint64_t)a.M, (uint64_t)a.r, (uint64_t)a.ldt, 128, (uint32_t)pl.swb / 2);
     else

@@ -177,7 +177,7 @@ lrd_status_t lrd_set_path(lrd_path_t path) {
 lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chunk_columns) {
     if (cluster_blocks != 0 && cluster_blocks != 1 && cluster_blocks != 2 && cluster_blocks != 4) return LRD_ERR_INVALID_ARG;
     if (kblocks_per_stage < 0 || kblocks_per_stage > 4) return LRD_ERR_INVALID_ARG;
-    if (chunk_columns != 0 && chunk_columns != 128 && chunk_columns != 192 && chunk_columns != 256) return LRD_ERR_INVALID_ARG;
+    if (chunk_columns != 0 && chunk_columns != 64 && chunk_columns != 128 && chunk_columns != 192 && chunk_columns != 256) return LRD_ERR_INVALID_ARG;
     chain_tuning(cluster_blocks, kblocks_per_stage, chunk_columns);
     return LRD_OK;
 }

@@ -108,6 +108,17 @@ lrd_tucker_freeze_t lrd_tucker_freeze_for_epoch(int64_t e);
  * gradient through but gets no weight gradient), as LRD_PLAN_* bits; 0 for a bad mask. */
 uint32_t lrd_linear_bwd_plan(lrd_freeze_t freeze);
 
+/* Algorithm 1 (rank search on a measured step-time curve), host only.  t[i] is the measured step time
+ * of the layer decomposed at rank R_min + i, i = 0 .. n-1 (so t[n-1] belongs to the starting rank R);
+ * T_orig is the step time of the undecomposed layer.  The paper's difference t(r) - t(r-1) refers, with
+ * r running downward, to a time not yet measured; the reading taken here: delta(r) = t(r+1) - t(r) for
+ * R_min <= r < R is the time saved by stepping down to r, R_opt is the first local maximum of delta met
+ * scanning down from R-1 (strictly above both neighbours and above zero; an end point has one neighbour),
+ * and with no such peak the global maximum (largest r on ties).  *use_decomposed (nullable) receives 1
+ * when t(R_opt) < T_orig (the algorithm's closing test: keep the original layer otherwise), else 0.
+ * Returns R_opt, or -(lrd_status_t) for a null curve, n < 1 or R_min < 1.  `t` is host memory. */
+int64_t lrd_rank_search(const double* t, int64_t n, int64_t R_min, double T_orig, int* use_decomposed);
+
 const char* lrd_status_string(lrd_status_t s);
 
 /* Process-wide choice of execution path (default LRD_PATH_AUTO).  Returns LRD_ERR_INVALID_ARG

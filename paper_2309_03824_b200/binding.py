@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_rank_search",
 ]
 
 
@@ -56,6 +56,8 @@ _lib.lrd_launch_count.restype = C.c_uint64
 _lib.lrd_launch_count.argtypes = []
 _lib.lrd_set_path.restype = _int
 _lib.lrd_set_path.argtypes = [_int]
+_lib.lrd_rank_search.restype = _i64
+_lib.lrd_rank_search.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double, C.POINTER(C.c_int)]
 _lib.lrd_chain_tuning.restype = _int
 _lib.lrd_chain_tuning.argtypes = [_int, _int, _int]
 _lib.lrd_check_device_status.restype = _int
@@ -129,6 +131,16 @@ def lrd_freeze_for_epoch(e):
 
 def lrd_tucker_freeze_for_epoch(e):
     return int(_lib.lrd_tucker_freeze_for_epoch(e))
+
+
+def lrd_rank_search(t, R_min, T_orig):
+    """Algorithm 1 on a measured curve: t[i] = step time at rank R_min + i.  Returns (R_opt, use_decomposed)."""
+    arr = (C.c_double * len(t))(*[float(x) for x in t])
+    use = C.c_int(0)
+    r = int(_lib.lrd_rank_search(arr, len(t), int(R_min), float(T_orig), C.byref(use)))
+    if r < 0:
+        raise LrdError(-r)
+    return r, bool(use.value)
 
 
 def lrd_linear_bwd_plan(freeze):

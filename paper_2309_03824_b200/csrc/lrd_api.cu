@@ -150,6 +150,32 @@ uint32_t lrd_linear_bwd_plan(lrd_freeze_t f) {
     return plan;
 }
 
+int64_t lrd_rank_search(const double* t, int64_t n, int64_t R_min, double T_orig, int* use_decomposed) {
+    if (!t || n < 1 || R_min < 1) return -(int64_t)LRD_ERR_INVALID_ARG;
+    int64_t best = -1;
+    if (n == 1) {
+        best = 0;
+    } else {
+        // delta[i] = t[i + 1] - t[i] belongs to rank R_min + i, i = 0 .. n-2
+        for (int64_t i = n - 2; i >= 0 && best < 0; --i) {
+            const double d = t[i + 1] - t[i];
+            const bool above_left = i == 0 || d > t[i] - t[i - 1];
+            const bool above_right = i == n - 2 || d > t[i + 2] - t[i + 1];
+            if (above_left && above_right && d > 0.0) best = i;
+        }
+        if (best < 0) {                                   // no peak: the global maximum, largest rank on ties
+            double mx = t[1] - t[0];
+            best = 0;
+            for (int64_t i = 1; i <= n - 2; ++i) {
+                const double d = t[i + 1] - t[i];
+                if (d >= mx) { mx = d; best = i; }
+            }
+        }
+    }
+    if (use_decomposed) *use_decomposed = t[best] < T_orig ? 1 : 0;
+    return R_min + best;
+}
+
 const char* lrd_status_string(lrd_status_t s) {
     switch (s) {
         case LRD_OK: return "ok";

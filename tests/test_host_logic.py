@@ -75,3 +75,31 @@ def test_argument_errors_are_reported_before_any_launch():
     with pytest.raises(b.LrdError):
         b.lrd_set_path(17)
     b.lrd_set_path(b.LRD_PATH_AUTO)
+
+
+def test_rank_search_bit_exact_against_oracle():
+    """Algorithm 1 on synthetic step-time curves: the library's host routine and the oracle pick the same rank
+    and take the same keep-the-original decision (staircases, ties, flat and monotone curves, one point)."""
+    import numpy as np
+    rng = np.random.default_rng(77)
+    curves = [np.array([1.0 if r <= 256 else 1.15 for r in range(250, 263)]), np.array([1.0, 1.0, 1.3, 1.3, 1.3, 1.4, 1.4]),
+              np.linspace(1.0, 2.0, 11), np.ones(9), np.array([3.0]), np.array([2.0, 1.0]), np.array([1.0, 2.0])]
+    for _ in range(300):
+        n = int(rng.integers(1, 40))
+        kind = int(rng.integers(0, 3))
+        if kind == 0:        # few distinct levels: many ties
+            curves.append(rng.integers(1, 5, size=n).astype(np.float64))
+        elif kind == 1:      # noisy rising curve with cliffs at multiples of 8
+            r = np.arange(n)
+            curves.append(1.0 + 0.01 * r + 0.2 * (r // 8) + 0.005 * rng.standard_normal(n))
+        else:
+            curves.append(rng.random(n))
+    for t in curves:
+        for T in (0.5, float(np.median(t)), 10.0):
+            want = o.rank_search(t, 100, T)
+            got = b.lrd_rank_search(t, 100, T)
+            assert got == want, (t, T, got, want)
+    with pytest.raises(b.LrdError):
+        b.lrd_rank_search([], 100, 1.0)
+    with pytest.raises(b.LrdError):
+        b.lrd_rank_search([1.0, 2.0], 0, 1.0)

@@ -73,6 +73,10 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // set-up above touched only this block's own shared and tensor memory: under programmatic dependent launch it
+    // overlaps the tail of the previous kernel in the stream; global memory is first touched below this line
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp == 0) {
         // TMA producer: the whole warp runs the loop, one elected lane issues
@@ -220,6 +224,10 @@ filter_kernel(const __grid_constant__ CUtensorMap tmDout, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // set-up above touched only this block's own shared and tensor memory: under programmatic dependent launch it
+    // overlaps the tail of the previous kernel in the stream; global memory is first touched below this line
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp == 0) {
         int s = 0;
@@ -338,6 +346,23 @@ int filter_splits(int64_t B, const Geo& g, int64_t ci, int64_t co) {
     return (int)((chunks + per - 1) / per);
 }
 
+// Launch with the programmatic-serialization attribute: the kernel waits (griddepcontrol.wait) before it
+// touches global memory, so its set-up may overlap the previous kernel's tail.
+template <typename K, typename... Args>
+void launch_pdl(K kern, dim3 grid, uint32_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kern, args...);     // errors surface through cudaGetLastError() at the call site
+}
+
 template <typename K>
 bool set_smem(K kern, uint32_t bytes) {
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
@@ -378,8 +403,8 @@ lrd_status_t tc_conv3x3(bool dgrad, const void* img, const void* G, void* out, i
         configured = true;
     }
     dim3 grid((unsigned)((n_total + 127) / 128), (unsigned)g.tiles_per_img, (unsigned)B);
-    if (dgrad) conv_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(tImg, tG, p);
-    else conv_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(tImg, tG, p);
+    if (dgrad) launch_pdl(conv_kernel<true>, grid, kSmemBytes, s, tImg, tG, p);
+    else launch_pdl(conv_kernel<false>, grid, kSmemBytes, s, tImg, tG, p);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
@@ -407,7 +432,7 @@ lrd_status_t tc_conv3x3_filter(const void* dout, const void* in, void* dG, int64
         configured = true;
     }
     dim3 grid(9, (unsigned)(((co + 127) / 128) * p.tiles_i), (unsigned)splits);
-    filter_kernel<<<grid, kThreads, kFSmemBytes, s>>>(tD, tI, p);
+    launch_pdl(filter_kernel, grid, kFSmemBytes, s, tD, tI, p);
     const int64_t n = co * 9 * ci;
     filter_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(scratch, splits, (int)co, (int)ci, p.ldp, (__nv_bfloat16*)dG);
     count_launch(2);

@@ -2,19 +2,21 @@
 //
 // A cluster of C blocks owns one 128-row tile.
 //   Phase 1  block c forms its r/C-column slice of T = In P in tensor memory (TMA-fed tcgen05.mma:
-//            In K-major, the slice of P MN-major).  The whole dynamic shared memory is the ring of
-//            this phase: many small stages, so that nearly all of it is in flight at any time.
+//            In K-major, the slice of P MN-major), one or two 64-deep k-blocks per stage, as many
+//            stages as the shared memory beside the T buffer holds.
 //   Gather   four warps read the slice (tcgen05.ld), round it to bf16 and write it into this block's T
 //            buffer (K-major, swizzled, slices are whole atoms = one contiguous range); one thread then
 //            copies the range into every peer's T buffer with bulk DSMEM copies that complete on the
-//            peer's barrier.  The T buffer lies over ring space of phase 1, so a block pushes only after
-//            every block of the cluster has reported the end of its phase-1 MMAs.  T never goes to
-//            global memory unless T_save asks.
+//            peer's barrier.  T never goes to global memory unless T_save asks.
 //   Phase 2  block c forms every C-th column chunk of Out = T Q^T (T from shared memory, Q by TMA, one
-//            64-deep tile per stage), double-buffered in tensor memory; the epilogue adds the bias,
-//            rounds to bf16 and leaves through [128 x 64] shared-memory slabs by TMA stores (which
-//            clip the ragged edges).
+//            64-deep tile per stage), double-buffered in tensor memory; each epilogue warp adds the
+//            bias (staged in shared memory while the MMAs run), rounds to bf16 and stores its 32 rows
+//            through its own [32 x 32] slabs by TMA stores (which clip the ragged edges).
 // Warp 0: TMA producer.  Warp 1: tensor memory + MMA issue.  Warps 2-5: gather and epilogue.
+// Two cluster barriers: the first (every block's barriers exist) is arrived at once and waited on only
+// where the first remote copy is near; the second (every block has received all slices sent to it) lets
+// no block leave while a peer may still be reading its shared memory.  The kernel's set-up runs before
+// griddepcontrol.wait and so overlaps the tail of the previous kernel in the stream.
 // Every wait is bounded; a wait that runs out raises the device timeout flag and the block tears
 // down in order.
 #include "chain.cuh"

@@ -13,9 +13,9 @@
 //
 // One 128 x BN output tile per block.  Warp 0 issues TMA loads, warp 1 owns tensor memory and
 // issues the MMAs, warps 2-5 read the accumulator (each its own quarter of the 128 lanes) and
-// store.  The single-thread instructions are issued under elect.sync by a converged warp.  Both operands may be K-major (reduction index contiguous) or MN-major (row / column
-// index contiguous), which covers every product of the forward and backward pass without a
-// transposed copy.
+// store.  The single-thread instructions are issued under elect.sync by a converged warp.  Both
+// operands may be K-major (reduction index contiguous) or MN-major (row / column index contiguous),
+// which covers every product of the forward and backward pass without a transposed copy.
 #include <algorithm>
 
 #include "common.cuh"
@@ -477,8 +477,9 @@ bool tc_gemm_eligible(const GemmArgs& g) {
     return true;
 }
 
-// Tile width.  One k-block of a 128 x BN tile costs four MMAs of max(77, BN / 2) cycles each (an MMA
-// narrower than 154 columns is issue-bound), so a 64-wide tile is as slow as a 128-wide one.
+// Tile width.  Every MMA of a tile reads its 128 x 16 block of A from shared memory whatever its width, and
+// every tile streams its own copy of A, so a narrow tile pays the same A traffic for fewer columns: below
+// about 154 columns the cost of a k-block is taken as constant, above as proportional to the width.
 //   split = false: blocks run in waves over the SMs -> minimise waves x per-tile cost;
 //   split = true:  the reduction is split until the machine is full -> minimise tiles x per-tile cost.
 static int pick_bn(int64_t M, int64_t N, bool split) {

@@ -70,6 +70,11 @@ lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void*
     void* Z1 = Z1_save ? Z1_save : ws;
     void* Z2 = Z2_save ? Z2_save : (void*)((uint8_t*)ws + act_bytes(t, t.r1));
     LRD_TRY(run_gemm(make_gemm(t.P, t.r1, t.C, X, t.C, false, A, t.r1, true, Z1, t.r1, nullptr, t.dt), path, false, nullptr, 0, s));
+    // core + last 1x1 in one launch where the shape allows: Z2 then stays on chip unless the caller saves it
+    if ((path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+        tc_conv_chain_eligible(false, t.B, t.H, t.W, t.r1, t.r2, t.S, t.dt, Z1, G, Bm, Y, Z2_save) &&
+        (!bias || ((uintptr_t)bias % 2) == 0))
+        return tc_conv3x3_chain(false, Z1, G, Bm, bias, Y, Z2_save, t.B, t.H, t.W, t.r1, t.r2, t.S, s);
     LRD_TRY(conv3x3_fwd(Z1, G, Z2, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
     return run_gemm(make_gemm(t.P, t.S, t.r2, Z2, t.r2, false, Bm, t.r2, false, Y, t.S, bias, t.dt), path, false, nullptr, 0, s);
 }
@@ -95,8 +100,12 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
     const size_t pbytes = ws_bytes - act_bytes(t, t.r1) - act_bytes(t, t.r2);
 
     LRD_TRY(run_gemm(make_gemm(t.P, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
-    if (dX || factors) LRD_TRY(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
-    if (dX) LRD_TRY(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
+    // transposed core + first 1x1 (dX = dZ1 A^T) in one launch where the shape allows; dZ1 is written only for dA
+    const bool fuse_dx = dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+                         tc_conv_chain_eligible(true, t.B, t.H, t.W, t.r1, t.r2, t.C, t.dt, dZ2, G, A, dX, factors ? dZ1 : nullptr);
+    if (fuse_dx) LRD_TRY(tc_conv3x3_chain(true, dZ2, G, A, nullptr, dX, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.r1, t.r2, t.C, s));
+    else if (dX || factors) LRD_TRY(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    if (dX && !fuse_dx) LRD_TRY(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
     if (factors) {
         GemmArgs gb = make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt);
         bool db_done = false;

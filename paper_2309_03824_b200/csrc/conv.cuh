@@ -31,6 +31,14 @@ bool tc_conv_eligible(int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, l
 size_t tc_conv_filter_scratch_bytes(int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co);
 lrd_status_t tc_conv3x3(bool dgrad, const void* img, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
                         int64_t co, cudaStream_t s);
+// The core followed by the 1x1 product that consumes it, in one launch (the core's result stays on chip unless
+// core_out asks for it): forward (dgrad = false) out2 = conv(img, G) Q^T + bias2 with Q = Bm [S x r2]; backward
+// (dgrad = true) out2 = conv^T(img, G) Q^T with Q = A [C x r1].  n2 = rows of Q = columns of out2 (<= 256).
+bool tc_conv_chain_eligible(bool dgrad, int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, int64_t n2, lrd_dtype_t dt,
+                            const void* img, const void* G, const void* Q, const void* out2, const void* core_out);
+lrd_status_t tc_conv3x3_chain(bool dgrad, const void* img, const void* G, const void* Q, const void* bias2, void* out2,
+                              void* core_out, int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, int64_t n2,
+                              cudaStream_t s);
 lrd_status_t tc_conv3x3_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W, int64_t ci,
                                int64_t co, float* scratch, size_t scratch_bytes, cudaStream_t s);
 

@@ -7,6 +7,12 @@
 //   conv_kernel<true> : data gradient  din[p][i] = sum_{tap,o} dout[p - tap][o] G[o][tap][i]
 //   filter_kernel     : filter gradient dG[o][tap][i] = sum_p dout[p][o] in[p + tap][i]   (split over
 //                       pixel chunks, fp32 partials added in a fixed order by filter_reduce_kernel)
+//   conv_kernel<.., true> (fused): the 1x1 product that follows the core runs in the same kernel.  The
+//                       tile of the core's result is rounded to bf16 into shared memory (K-major,
+//                       128-byte swizzle; written to memory only if the caller needs it), the ring,
+//                       dead by then, receives the 1x1 factor Q[N2 x n1], and a second set of MMAs forms
+//                       out2[p][:] = core[p][:] Q^T (+ bias) in other tensor-memory columns:
+//                       forward  Y = conv(Z1, G) Bm^T + b,  backward  dX = conv^T(dZ2, G) A^T.
 //
 // A tile is bh rows of one image (bh * W <= 128 pixels = the 128 MMA rows / the reduction chunk).
 // Warp roles as in the matrix-product kernel: TMA producer, MMA issuer (both issue under elect.sync from a converged warp), 4 epilogue warps.
@@ -33,16 +39,22 @@ struct ConvParams {
     int n_total;            // output channels of this product (columns of out)
     int g_ci;               // Ci of G[o][tap][i] (its row length is 9 * g_ci)
     int sign;               // +1 forward, -1 data gradient
-    __nv_bfloat16* out;     // [B*H*W][n_total]
+    __nv_bfloat16* out;     // [B*H*W][n_total]; fused: nullable (the core's result is then never written to memory)
     unsigned int* timeout_flag;
+    // fused 1x1 product
+    int n2;                       // columns of out2 (<= 256)
+    __nv_bfloat16* out2;          // [B*H*W][n2]
+    const __nv_bfloat16* bias2;   // [n2] or nullptr
 };
 
-// grid: (ceil(n_total / 128), tiles_per_img, B)
-template <bool DGRAD>
+// grid: (ceil(n_total / 128), tiles_per_img, B); fused: n_total <= 128, so gridDim.x = 1
+template <bool DGRAD, bool FUSE>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ CUtensorMap tmG, const ConvParams p) {
+conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ CUtensorMap tmG,
+            const __grid_constant__ CUtensorMap tmQ, const ConvParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], acc_bar;
+    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], acc_bar, q_full, t_ready, out_full;
+    constexpr uint32_t kTmemCols = FUSE ? 512 : 128;        // fused: the second product accumulates in columns [256, 512)
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -63,10 +75,14 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
             mbar_init(smem_u32(&empty_bar[s]), 1);
         }
         mbar_init(smem_u32(&acc_bar), 1);
+        mbar_init(smem_u32(&q_full), 1);
+        mbar_init(smem_u32(&t_ready), 4);
+        mbar_init(smem_u32(&out_full), 1);
+        if (FUSE) prefetch_tmap(&tmQ);
         fence_mbar_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&tmem_base_slot), 128);
+        tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -77,6 +93,10 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
     // overlaps the tail of the previous kernel in the stream; global memory is first touched below this line
     griddep_launch_dependents();
     griddep_wait();
+    // fused: once the core's MMAs are done the ring is dead; it then holds [T: 2 atoms of 128 rows x 64 columns |
+    // Q: one [256 rows x 64 k] tile per 64 columns of the core's result]
+    const uint32_t t_base = smem_base, q_base = smem_base + 2 * kTile;
+    const int nq = (p.n_total + 63) / 64;
 
     if (warp == 0) {
         // TMA producer: the whole warp runs the loop, one elected lane issues
@@ -101,6 +121,15 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
             }
             __syncwarp();
             if (++s == kStages) { s = 0; ph ^= 1; }
+        }
+        if (FUSE) {                                          // the 1x1 factor, into the dead ring (rows past n2, columns past n1: zeros)
+            if (mbar_wait_uniform(smem_u32(&acc_bar), 0, ab)) {
+                if (elect_one()) {
+                    mbar_expect_tx(smem_u32(&q_full), (uint32_t)nq * 2u * kTile);
+                    for (int kb = 0; kb < nq; ++kb) tma_load_2d(q_base + kb * 2 * kTile, &tmQ, smem_u32(&q_full), kb * 64, 0);
+                }
+                __syncwarp();
+            }
         }
     } else if (warp == 1) {
         // MMA issuer: converged warp, elect.sync around the issue
@@ -128,13 +157,30 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
         }
         if (ok && elect_one()) mma_commit(smem_u32(&acc_bar));
         __syncwarp();
+        if (FUSE) {                                          // out2 tile = T Q^T, reduction over the n_total columns of T
+            if (ok) ok = mbar_wait_uniform(smem_u32(&t_ready), 0, ab);
+            if (ok) ok = mbar_wait_uniform(smem_u32(&q_full), 0, ab);
+            if (ok) {
+                tc_fence_after();
+                const uint32_t idesc2 = idesc_bf16((p.n2 + 15) / 16 * 16, false, false);
+                if (elect_one()) {
+                    for (int ks = 0; ks * 16 < p.n_total; ++ks) {
+                        const uint64_t ad = smem_desc_sw128(t_base + (ks / 4) * kTile + (ks % 4) * 32, 0, 1024);
+                        const uint64_t bd = smem_desc_sw128(q_base + (ks / 4) * 2 * kTile + (ks % 4) * 32, 0, 1024);
+                        mma_bf16_ss(tmem_base + 256u, ad, bd, idesc2, ks > 0 ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&out_full));
+                }
+                __syncwarp();
+            }
+        }
     } else {
         const int q = warp % 4;
-        const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
+        const bool ready = mbar_wait_uniform(smem_u32(&acc_bar), 0, ab);
         tc_fence_after();
+        const int row = q * 32 + lane;                           // pixel of the tile: (h0 + row / W, row % W)
+        const bool row_ok = row < p.bh * p.W && h0 + row / p.W < p.H;
         if (ready) {
-            const int row = q * 32 + lane;                       // pixel of the tile: (h0 + row / W, row % W)
-            const bool row_ok = row < p.bh * p.W && h0 + row / p.W < p.H;
             __nv_bfloat16* dst_row = p.out + ((int64_t)(img * p.H + h0) * p.W + row) * p.n_total;
 #pragma unroll 1
             for (int cchunk = 0; cchunk < 4; ++cchunk) {
@@ -142,6 +188,20 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
                 tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + cchunk * 32, v);
                 tmem_ld_wait();
                 const int col0 = n0 + cchunk * 32;
+                if (FUSE) {                                  // bf16 tile T for the second product (rows past the tile hold
+                    if (col0 < p.n_total) {                  // garbage that only reaches output rows nobody stores)
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const uint32_t col = (uint32_t)(cchunk * 32 + g * 8);
+                            st_shared_v4(t_base + (col / 64u) * kTile + (uint32_t)row * 128u + ((((col % 64u) / 8u) ^ ((uint32_t)row & 7u)) << 4),
+                                         pack_bf16(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1])),
+                                         pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3])),
+                                         pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5])),
+                                         pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7])));
+                        }
+                    }
+                    if (!p.out) continue;
+                }
                 if (!row_ok || col0 >= p.n_total) continue;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
@@ -158,6 +218,57 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
                 }
             }
         }
+        if (FUSE) {
+            fence_proxy_async_smem();                        // T was written by ordinary stores, the MMA reads it through the async proxy
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&t_ready));
+            const bool done = ready && mbar_wait_uniform(smem_u32(&out_full), 0, ab);
+            tc_fence_after();
+            if (done) {
+                __nv_bfloat16* dst_row = p.out2 + ((int64_t)(img * p.H + h0) * p.W + row) * p.n2;
+                const bool bias_vec = p.bias2 && (((uintptr_t)p.bias2 & 15u) == 0);
+#pragma unroll 1
+                for (int cchunk = 0; cchunk * 32 < p.n2; ++cchunk) {
+                    const int col0 = cchunk * 32;
+                    uint4 bv[4] = {};
+                    const bool bvec = bias_vec && col0 + 32 <= p.n2;
+                    if (bvec) {
+                        const uint4* bp = reinterpret_cast<const uint4*>(p.bias2 + col0);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) bv[e] = __ldg(bp + e);
+                    }
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + 256u + ((uint32_t)(q * 32) << 16) + cchunk * 32, v);
+                    tmem_ld_wait();
+                    if (!row_ok) continue;
+                    if (bvec) {
+                        const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            v[2 * e] = __float_as_uint(__uint_as_float(v[2 * e]) + __uint_as_float(bw[e] << 16));
+                            v[2 * e + 1] = __float_as_uint(__uint_as_float(v[2 * e + 1]) + __uint_as_float(bw[e] & 0xFFFF0000u));
+                        }
+                    } else if (p.bias2) {
+                        for (int e = 0; e < 32; ++e)
+                            if (col0 + e < p.n2) v[e] = __float_as_uint(__uint_as_float(v[e]) + __bfloat162float(p.bias2[col0 + e]));
+                    }
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (col0 + g * 8 + 8 <= p.n2) {
+                            *reinterpret_cast<uint4*>(dst_row + col0 + g * 8) =
+                                make_uint4(pack_bf16(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1])),
+                                           pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3])),
+                                           pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5])),
+                                           pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7])));
+                        } else {
+                            for (int e = 0; e < 8; ++e)
+                                if (col0 + g * 8 + e < p.n2) dst_row[col0 + g * 8 + e] = __float2bfloat16_rn(__uint_as_float(v[8 * g + e]));
+                        }
+                    }
+                }
+            }
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -165,7 +276,7 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
         if (abort_flag)
             for (int i = 0; i < 256; ++i) __nanosleep(1000);
         tc_fence_after();
-        tmem_dealloc(tmem_base, 128);
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -397,14 +508,53 @@ lrd_status_t tc_conv3x3(bool dgrad, const void* img, const void* G, void* out, i
     p.B = (int)B; p.H = (int)H; p.W = (int)W; p.bh = g.bh; p.tiles_per_img = g.tiles_per_img;
     p.ka = (int)ka; p.n_total = (int)n_total; p.g_ci = (int)ci; p.sign = dgrad ? -1 : 1;
     p.out = (__nv_bfloat16*)out; p.timeout_flag = device_timeout_flag();
+    p.n2 = 0; p.out2 = nullptr; p.bias2 = nullptr;
     static bool configured = false;
     if (!configured) {
-        if (!set_smem(conv_kernel<false>, kSmemBytes) || !set_smem(conv_kernel<true>, kSmemBytes)) return LRD_ERR_CUDA;
+        if (!set_smem(conv_kernel<false, false>, kSmemBytes) || !set_smem(conv_kernel<true, false>, kSmemBytes)) return LRD_ERR_CUDA;
         configured = true;
     }
     dim3 grid((unsigned)((n_total + 127) / 128), (unsigned)g.tiles_per_img, (unsigned)B);
-    if (dgrad) launch_pdl(conv_kernel<true>, grid, kSmemBytes, s, tImg, tG, p);
-    else launch_pdl(conv_kernel<false>, grid, kSmemBytes, s, tImg, tG, p);
+    if (dgrad) launch_pdl(conv_kernel<true, false>, grid, kSmemBytes, s, tImg, tG, tG, p);
+    else launch_pdl(conv_kernel<false, false>, grid, kSmemBytes, s, tImg, tG, tG, p);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+bool tc_conv_chain_eligible(bool dgrad, int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, int64_t n2, lrd_dtype_t dt,
+                            const void* img, const void* G, const void* Q, const void* out2, const void* core_out) {
+    const int64_t n1 = dgrad ? ci : co;                  // channels of the core's result = reduction of the 1x1 product
+    if (!tc_conv_eligible(B, H, W, ci, co, dt, img, G, Q)) return false;
+    if (n1 > 128 || n1 % 16 || n2 < 8 || n2 > 256 || n2 % 8) return false;
+    return a16(out2) && (!core_out || a16(core_out));
+}
+
+// The core followed by the 1x1 product out2[p][:] = core[p][:] Q^T (+ bias2) in one launch.  Q is [n2 x n1] with n1
+// contiguous; core_out (nullable) receives the core's bf16 result when the caller needs it later.
+lrd_status_t tc_conv3x3_chain(bool dgrad, const void* img, const void* G, const void* Q, const void* bias2, void* out2,
+                              void* core_out, int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, int64_t n2,
+                              cudaStream_t s) {
+    Geo g;
+    if (!geometry(B, H, W, ci, co, &g)) return LRD_ERR_UNSUPPORTED;
+    const int64_t ka = dgrad ? co : ci, n1 = dgrad ? ci : co;
+    CUtensorMap tImg, tG, tQ;
+    bool ok = make_tmap_nhwc_bf16(&tImg, img, (uint64_t)B, (uint64_t)H, (uint64_t)W, (uint64_t)ka, (uint32_t)g.bh, (uint32_t)W, 64);
+    ok = ok && make_tmap_2d_bf16(&tG, G, (uint64_t)co, (uint64_t)(9 * ci), (uint64_t)(9 * ci), dgrad ? 64 : 128, 64);
+    ok = ok && make_tmap_2d_bf16(&tQ, Q, (uint64_t)n2, (uint64_t)n1, (uint64_t)n1, 256, 64);
+    if (!ok) return LRD_ERR_CUDA;
+    ConvParams p;
+    p.B = (int)B; p.H = (int)H; p.W = (int)W; p.bh = g.bh; p.tiles_per_img = g.tiles_per_img;
+    p.ka = (int)ka; p.n_total = (int)n1; p.g_ci = (int)ci; p.sign = dgrad ? -1 : 1;
+    p.out = (__nv_bfloat16*)core_out; p.timeout_flag = device_timeout_flag();
+    p.n2 = (int)n2; p.out2 = (__nv_bfloat16*)out2; p.bias2 = (const __nv_bfloat16*)bias2;
+    static bool configured = false;
+    if (!configured) {
+        if (!set_smem(conv_kernel<false, true>, kSmemBytes) || !set_smem(conv_kernel<true, true>, kSmemBytes)) return LRD_ERR_CUDA;
+        configured = true;
+    }
+    dim3 grid(1, (unsigned)g.tiles_per_img, (unsigned)B);
+    if (dgrad) launch_pdl(conv_kernel<true, true>, grid, kSmemBytes, s, tImg, tG, tQ, p);
+    else launch_pdl(conv_kernel<false, true>, grid, kSmemBytes, s, tImg, tG, tQ, p);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }

@@ -65,7 +65,8 @@ def test_general_path_small_geometries(dtype, geom, freeze):
     check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, dtype, 400 + H), freeze, path=b.LRD_PATH_GENERAL)
 
 
-@pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 9, 11, 128, 136, 96, 104), (5, 14, 14, 256, 256, 96, 96)])
+@pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 9, 11, 128, 136, 96, 104), (5, 14, 14, 256, 256, 96, 96),
+                                  (3, 10, 12, 72, 200, 48, 64), (2, 7, 9, 40, 24, 16, 16), (1, 14, 14, 256, 248, 128, 112)])
 @pytest.mark.parametrize("freeze", MASKS)
 def test_tensor_core_path(geom, freeze):
     B, H, W, C, S, r1, r2 = geom

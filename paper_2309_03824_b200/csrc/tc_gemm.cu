@@ -198,7 +198,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
         tc_fence_after();
         if (warp == 2 && lane == 0) { LRD_TS(6); }
-        cluster_arrive();      // barrier 1: this block's pipeline ring is dead (all its MMAs have completed)
+        // barrier 1: this block's pipeline ring is dead (all its MMAs have completed).  Progress only: what the peers
+        // must see of this block (its initialised barriers) is released by the arrivals of warps 0 and 1.
+        cluster_arrive_relaxed();
+        if (warp == 2 && lane == 0) { LRD_TS(13); }
         if (ok) {
             // partial tile -> staging, laid out [owner][row][cs] so that each owner's slice is one contiguous range
             const bool has_work = kb_begin < kb_end;       // a block past the end of the reduction contributes zeros
@@ -260,6 +263,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (warp == 2 && lane == 0) { LRD_TS(10); }
         cluster_arrive_relaxed();   // barrier 2: everything addressed to this block has landed (progress only, no data)
+        if (warp == 2 && lane == 0) { LRD_TS(14); }
         if (ok) {
             // this block's column slice: add the S partials in rank order, round once, store
             const int64_t grow = (int64_t)m0 + row;
@@ -295,6 +299,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
+            if (warp == 2 && lane == 0) { LRD_TS(15); }
             if (with_colsum && self == 0 && p.colsum_out && grow < p.M) {
                 float t = 0.f;
                 for (uint32_t k = 0; k < S; ++k) {

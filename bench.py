@@ -361,11 +361,23 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
+        t_wait = time.time()
+        while not sampler.rows and time.time() - t_wait < 5.0:      # nvidia-smi takes a moment to print its first sample
+            time.sleep(0.05)
     for i in range(args.warmup):
         step(i)
     ms, t0, t1 = timed(step, args.steps)
-    clocks = sampler.summary(t0, t1) if rank == 0 else None
+    # The timed region is shorter than one sampling period (K steps of ~0.2 ms): the same steps go on, untimed, for
+    # about a second and a half so that the clock samples are taken under this very load.
+    if rank == 0:
+        i = args.steps
+        while time.time() - t1 < 1.5:
+            for _ in range(100):
+                step(i)
+                i += 1
+            torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.summary(t0, time.time()) if rank == 0 else None
     ms_per_step = ms / args.steps
     tokens = wl.C1_M * world
     value = whole_job_value(wl.C1_M, world, ms_per_step)

@@ -477,6 +477,7 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         int G1 = g_tune_G1 ? g_tune_G1 : (kb1 <= 16 ? 2 : 1);
         if (G1 > 4) G1 = 4;
         if (G1 > kb1) G1 = kb1;
+        while (!g_tune_G1 && G1 > 1 && ring1 < 2 * (int64_t)G1 * kb1_bytes) --G1;   // a wide T buffer leaves room for single k-blocks only
         if (ring1 < 2 * (int64_t)G1 * kb1_bytes) continue;
         int S1 = (int)(ring1 / ((int64_t)G1 * kb1_bytes)), S2 = (int)(ring2 / (int64_t)kb2_bytes);
         if (S1 > kMaxStages) S1 = kMaxStages;
@@ -505,6 +506,17 @@ void chain_tuning(int C, int G1, int BN2) {
 bool chain_eligible(const ChainArgs& a) {
     Plan pl;
     return make_plan(a, &pl);
+}
+
+// The fused kernel loses to two separate products where the T buffer (128 rows x r) leaves room for only two
+// phase-1 stages and the first reduction is long (measured: r = 512 with K1 = 4096, where every block also re-reads
+// a 1 MB activation tile: 99 us fused against 57 us unfused at 8192 tokens).  The automatic path then takes the
+// separate products; LRD_PATH_FUSED still forces the chain.
+bool chain_preferred(const ChainArgs& a) {
+    Plan pl;
+    if (!make_plan(a, &pl)) return false;
+    const int64_t kb1 = (a.K1 + 63) / 64;
+    return !(pl.S1 <= 2 && kb1 > 32);
 }
 
 lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {

@@ -22,6 +22,8 @@ struct ChainArgs {
 // phase-2 chunk width.  0 = automatic.  Not thread-safe against concurrent launches.
 void chain_tuning(int C, int G1, int BN2);
 bool chain_eligible(const ChainArgs& c);
+// Eligible, and expected to beat the two separate products (the automatic path's test).
+bool chain_preferred(const ChainArgs& c);
 lrd_status_t chain_launch(const ChainArgs& c, cudaStream_t stream);
 
 }  // namespace lrd

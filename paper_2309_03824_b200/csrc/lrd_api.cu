@@ -256,7 +256,7 @@ lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const 
         c.M = L.M; c.K1 = L.K; c.r = L.r; c.N2 = L.N;
         c.In = X; c.ld_in = L.ldx; c.P = V; c.ldp = L.ldv; c.Q = U; c.ldq = L.ldu; c.bias = bias;
         c.Out = Y; c.ld_out = L.ldy; c.T_save = Z_save; c.ldt = L.ldz; c.dtype = L.dt;
-        if (chain_eligible(c)) return chain_launch(c, s);
+        if (path == LRD_PATH_FUSED ? chain_eligible(c) : chain_preferred(c)) return chain_launch(c, s);
     }
     void* Z = Z_save ? Z_save : workspace;
     const int64_t ldz = Z_save ? L.ldz : L.r;
@@ -305,7 +305,7 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
         c.M = L.M; c.K1 = L.N; c.r = L.r; c.N2 = L.K;
         c.In = dY; c.ld_in = L.ldy; c.P = U; c.ldp = L.ldu; c.Q = V; c.ldq = L.ldv; c.bias = nullptr;
         c.Out = dX; c.ld_out = L.ldx; c.T_save = need_dz_in_memory ? dZ : nullptr; c.ldt = L.r; c.dtype = L.dt;
-        if (chain_eligible(c)) {
+        if (path == LRD_PATH_FUSED ? chain_eligible(c) : chain_preferred(c)) {
             LRD_TRY(chain_launch(c, s));
             chained = true;
         }

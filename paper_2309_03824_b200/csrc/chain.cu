@@ -509,14 +509,13 @@ bool chain_eligible(const ChainArgs& a) {
 }
 
 // The fused kernel loses to two separate products where the T buffer (128 rows x r) leaves room for only two
-// phase-1 stages and the first reduction is long (measured: r = 512 with K1 = 4096, where every block also re-reads
-// a 1 MB activation tile: 99 us fused against 57 us unfused at 8192 tokens).  The automatic path then takes the
-// separate products; LRD_PATH_FUSED still forces the chain.
+// k-blocks of phase 1 in flight, i.e. at r = 512 (measured at 8192 tokens: 1024 -> 4096 forward 65 us fused against 49 us on two
+// persistent products, 4096 -> 1024 99 against 46 us; at r <= 384 the chain wins everywhere measured).  The
+// automatic path then takes the separate products; LRD_PATH_FUSED still forces the chain.
 bool chain_preferred(const ChainArgs& a) {
     Plan pl;
     if (!make_plan(a, &pl)) return false;
-    const int64_t kb1 = (a.K1 + 63) / 64;
-    return !(pl.S1 <= 2 && kb1 > 32);
+    return pl.S1 * pl.G1 > 2;          // k-blocks of phase 1 in flight
 }
 
 lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {

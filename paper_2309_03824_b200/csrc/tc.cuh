@@ -14,6 +14,9 @@ int tc_pick_splits(int64_t M, int64_t N, int64_t K);
 size_t tc_split_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // True when tc_gemm can also deliver g.a_colsum for this product (bf16, both operands MN-major, aligned).
 bool tc_gemm_colsum_ok(const GemmArgs& g);
+// Unsplit product with a bf16 result on the persistent kernel (one block per SM walks over the tiles, the
+// epilogue of a tile overlaps the MMAs of the next).  Same eligibility as tc_gemm; no column sums.
+lrd_status_t tc_gemm_persistent(const GemmArgs& g, cudaStream_t stream);
 // allow_split: the reduction dimension may be split over blocks (weight gradients).
 lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes, cudaStream_t stream);
 

@@ -603,6 +603,7 @@ lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_
     if (!tc_gemm_eligible(g)) return LRD_ERR_UNSUPPORTED;
     const bool ones = g.a_colsum != nullptr;
     if (ones && !tc_gemm_colsum_ok(g)) return LRD_ERR_UNSUPPORTED;
+    if (!allow_split && !ones) return tc_gemm_persistent(g, stream);   // data products: the persistent kernel
     int splits = 1, cluster = 1, bn;
     if (allow_split) {
         const SplitPlan sp = pick_split(g.M, g.N, g.K, ones);

@@ -260,16 +260,18 @@ lrd_status_t launch_p_major(bool a_mn, bool b_mn, const CUtensorMap& tA, const C
     return b_mn ? launch_p<BN, false, true>(tA, tB, tC, p, blocks, s) : launch_p<BN, false, false>(tA, tB, tC, p, blocks, s);
 }
 
-// Tile width: the widest that does not waste more than a quarter of its columns; 64 only for N <= 64.
-int pick_bn_p(int64_t N) {
+// Tile width: every block streams (A tile + B tile) per k-block and the slowest block walks over
+// ceil(tiles / SMs) tiles, so minimise that product; wider tiles on ties (fewer re-reads of A).
+int pick_bn_p(int64_t M, int64_t N) {
     if (N <= 64) return 64;
-    const int cands[3] = {256, 192, 128};
+    const int64_t mt = (M + BM - 1) / BM;
+    const int cands[4] = {256, 192, 128, 64};
     int best = 128;
-    double best_waste = 1e9;
+    double best_cost = 1e300;
     for (int bn : cands) {
-        const int64_t nt = (N + bn - 1) / bn;
-        const double waste = (double)(nt * bn - N) / (double)(nt * bn);
-        if (waste < best_waste - 0.05) { best_waste = waste; best = bn; }
+        const int64_t tiles = mt * ((N + bn - 1) / bn);
+        const double cost = (double)((tiles + kNumSms - 1) / kNumSms) * (double)(kATile + bn * BK * 2);
+        if (cost < best_cost) { best_cost = cost; best = bn; }
     }
     return best;
 }
@@ -278,7 +280,7 @@ int pick_bn_p(int64_t N) {
 
 lrd_status_t tc_gemm_persistent(const GemmArgs& g, cudaStream_t stream) {
     if (!tc_gemm_eligible(g) || g.a_colsum) return LRD_ERR_UNSUPPORTED;
-    const int bn = pick_bn_p(g.N);
+    const int bn = pick_bn_p(g.M, g.N);
     CUtensorMap tA, tB, tC;
     bool ok = g.a_mn_major ? make_tmap_2d_bf16(&tA, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, 64)
                            : make_tmap_2d_bf16(&tA, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda, BM, BK);

@@ -20,3 +20,14 @@ def test_rank_search_on_measured_curve_matches_oracle():
     assert (r_opt, use) == want
     assert R_min <= r_opt < R or R == R_min
     assert b.lrd_check_device_status() == b.LRD_OK
+
+
+def test_tucker_rank_search_on_measured_curve_matches_oracle():
+    B, H, C, S = 2, 6, 48, 64
+    R, R_min = rs.tucker_rank(C, S, 3, 2), rs.tucker_rank(C, S, 3, 3)
+    assert (R, R_min) == (o.tucker_rank(C, S, 3, 2)[0], o.tucker_rank_min(C, S, 3, 2)) and R_min < R
+    r_opt, curve = rs.search_tucker(B, H, H, C, S, R, R_min, iters=3)
+    assert sorted(curve) == list(range(R_min, R + 1)) and all(v > 0 for v in curve.values())
+    want, _ = o.rank_search([curve[r] for r in range(R_min, R + 1)], R_min, float("inf"))
+    assert r_opt == want and R_min <= r_opt <= R
+    assert b.lrd_check_device_status() == b.LRD_OK

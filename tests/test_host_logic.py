@@ -103,3 +103,15 @@ def test_rank_search_bit_exact_against_oracle():
         b.lrd_rank_search([], 100, 1.0)
     with pytest.raises(b.LrdError):
         b.lrd_rank_search([1.0, 2.0], 0, 1.0)
+
+
+def test_rank_formulas_of_the_search_driver_match_the_oracle():
+    """The driver's own Eq. 5 / Eq. 6 and its fully-connected analogue against the oracle's, on a grid; and the
+    paper's worked example."""
+    from paper_2309_03824_b200 import rank_search as rs        # imports torch, makes no CUDA call at import
+    assert rs.tucker_rank(512, 512, 3, 2) == 309 and rs.tucker_rank(512, 512, 3, 3) == o.tucker_rank_min(512, 512, 3, 2)
+    for C in (16, 64, 96, 256, 512, 2048):
+        for S in (16, 48, 256, 512, 1024):
+            for alpha in (2, 3, 4, 8):
+                assert rs.tucker_rank(C, S, 3, alpha) == max(o.tucker_rank(C, S, 3, alpha)[0], 1), (C, S, alpha)
+                assert rs.fc_rank(C, S, alpha) == max(o.svd_rank(C, S, alpha), 1), (C, S, alpha)

@@ -132,6 +132,14 @@ lrd_status_t lrd_set_path(lrd_path_t path);
  * thread-safe against concurrent launches.  Returns LRD_ERR_INVALID_ARG for values outside the lists. */
 lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chunk_columns);
 
+/* Launch-shape override of the unsplit products (the dense layer's forward and input gradient, the two
+ * products of an unfused decomposed layer), for measurement sweeps (no counterpart in the paper):
+ * blocks per MMA, 1 (every SM works on its own 128-row tiles) or 2 (pairs of SMs share 256-row tiles and
+ * each loads half of the B operand); 0 = automatic (the default).  2 is ignored for products of at most
+ * 128 rows.  Process-wide, not thread-safe against concurrent launches.  Returns LRD_ERR_INVALID_ARG for
+ * other values. */
+lrd_status_t lrd_gemm_tuning(int blocks_per_mma);
+
 /* Synchronises the current device, then reports and clears the device-side timeout flag:
  * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
 lrd_status_t lrd_check_device_status(void);

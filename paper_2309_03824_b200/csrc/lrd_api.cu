@@ -208,6 +208,12 @@ lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chu
     return LRD_OK;
 }
 
+lrd_status_t lrd_gemm_tuning(int blocks_per_mma) {
+    if (blocks_per_mma < 0 || blocks_per_mma > 2) return LRD_ERR_INVALID_ARG;
+    tc_gemm_persistent_force_pairs(blocks_per_mma);
+    return LRD_OK;
+}
+
 lrd_status_t lrd_check_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return LRD_ERR_CUDA;
     bool raised = false;

@@ -17,6 +17,7 @@ bool tc_gemm_colsum_ok(const GemmArgs& g);
 // Unsplit product with a bf16 result on the persistent kernel (one block per SM walks over the tiles, the
 // epilogue of a tile overlaps the MMAs of the next).  Same eligibility as tc_gemm; no column sums.
 lrd_status_t tc_gemm_persistent(const GemmArgs& g, cudaStream_t stream);
+void tc_gemm_persistent_force_pairs(int blocks_per_mma);     // 0: automatic; 1 or 2: forced where the shape allows
 // allow_split: the reduction dimension may be split over blocks (weight gradients).
 lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_t partial_bytes, cudaStream_t stream);
 

@@ -8,8 +8,15 @@
 // second product of an unfused decomposed layer) is otherwise all epilogue.
 // Warp 0: TMA producer.  Warp 1: tensor memory + MMA issue.  Warps 2-5: epilogue.  Single-thread
 // instructions are issued under elect.sync by a converged warp; every wait is bounded.
+//
+// CG = 2 runs the same loop on pairs of blocks (a cluster of two SMs, tcgen05 cta_group::2): a pair owns a
+// 256 x BN tile, each block loads its own 128 rows of A but only HALF of the B tile, and the even block
+// issues MMAs of 256 rows that read both halves.  Per k-block a block then takes (16 KB + BN x 64 B)
+// instead of (16 KB + BN x 128 B) through its L2 -> shared-memory path, which is what bounds the wide
+// tiles: at BN = 256 the shared-memory port sees 64 KB (fill + operand reads) per 512 MMA cycles instead
+// of 96 KB.
 #include "common.cuh"
-#include "ptx.cuh"
+#include "ptx_pair.cuh"
 #include "tc.cuh"
 #include "tma.cuh"
 
@@ -24,14 +31,21 @@ constexpr uint32_t kATile = BM * BK * 2;
 constexpr uint32_t kSlabBytes = 32 * 32 * 2;                 // one warp's slab: 32 rows x 32 columns of bf16
 constexpr uint32_t kStagingBytes = 4 * 2 * kSlabBytes;
 
-template <int BN> struct PCfg {
-    static constexpr uint32_t STAGE_BYTES = kATile + BN * BK * 2;
+template <int BN, int CG> struct PCfg {
+    static constexpr int BNH = BN / CG;                      // columns of B this block loads
+    static constexpr uint32_t STAGE_BYTES = kATile + BNH * BK * 2;
     static constexpr int STAGES_RAW = (200 * 1024) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
     static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + kStagingBytes + 1024;
     static constexpr uint32_t TMEM_COLS = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);
     static constexpr uint32_t BUF_COLS = TMEM_COLS / 2;      // column offset of the second accumulator
 };
+
+template <int CG>
+__device__ __forceinline__ void load2d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int x, int y) {
+    if (CG == 2) tma_load_2d_pair(dst, m, bar, x, y);        // bar: shared::cluster address (the even block's barrier)
+    else tma_load_2d(dst, m, bar, x, y);
+}
 
 struct PParams {
     int64_t M, N;
@@ -40,11 +54,14 @@ struct PParams {
     unsigned int* timeout_flag;
 };
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                           const __grid_constant__ CUtensorMap tmC, const PParams p) {
-    using C = PCfg<BN>;
+    using C = PCfg<BN, CG>;
+    constexpr int BNH = C::BNH;
+    static_assert(CG == 1 || CG == 2, "blocks per MMA");
+    static_assert(CG == 1 || !B_MN || BNH % 64 == 0, "an MN-major half of B is made of 64-column boxes");
     constexpr int STAGES = C::STAGES;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], out_full[2], out_empty[2];
@@ -55,7 +72,9 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     const uint32_t staging_base = smem_base, ring_base = smem_base + kStagingBytes;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
     const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
-    const int n_tiles_total = p.m_tiles * p.n_tiles;
+    const int n_tiles_total = p.m_tiles * p.n_tiles;         // p.m_tiles counts row tiles of 128 CG rows
+    const int h = CG == 2 ? (int)cluster_ctarank() : 0;      // this block's half of the pair
+    const int unit = (int)blockIdx.x / CG, n_units = (int)gridDim.x / CG;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -68,16 +87,26 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&out_full[i]), 1);
-            mbar_init(smem_u32(&out_empty[i]), 4);
+            mbar_init(smem_u32(&out_empty[i]), 4 * CG);       // the epilogue warps of every block of the pair
         }
         fence_mbar_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS);
-        tmem_relinquish();
+        if (CG == 2) {
+            tmem_alloc_pair(smem_u32(&tmem_base_slot), C::TMEM_COLS);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
-    __syncthreads();
+    if (CG == 2) {                   // the other block's barriers exist before anything signals them
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     // set-up above touched only this block's own shared and tensor memory: it may overlap the tail of the
@@ -90,40 +119,42 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         int s = 0;
         uint32_t ph = 1;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
-            const int m0 = (t % p.m_tiles) * BM, n0 = (t / p.m_tiles) * BN;
+        for (int t = unit; t < n_tiles_total && ok; t += n_units) {
+            const int m0 = (t % p.m_tiles) * (BM * CG) + h * BM, n0 = (t / p.m_tiles) * BN + h * BNH;
             for (int kb = 0; kb < p.kb_total; ++kb) {
                 ok = mbar_wait_uniform(smem_u32(&empty_bar[s]), ph, ab);
                 if (!ok) break;
-                const uint32_t fb = smem_u32(&full_bar[s]);
+                // a pair's loads all complete on the even block's barrier, which its MMA warp waits on
+                const uint32_t fb_local = smem_u32(&full_bar[s]);
+                const uint32_t fb = CG == 2 ? map_to_cta(fb_local, 0) : fb_local;
                 const uint32_t a_dst = ring_base + s * C::STAGE_BYTES, b_dst = a_dst + kATile;
                 const int k0 = kb * BK;
                 if (elect_one()) {
-                    mbar_expect_tx(fb, C::STAGE_BYTES);
+                    if (h == 0) mbar_expect_tx(fb_local, CG * C::STAGE_BYTES);
                     if (A_MN) {
 #pragma unroll
-                        for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * 8192, &tmA, fb, m0 + 64 * j, k0);
+                        for (int j = 0; j < BM / 64; ++j) load2d<CG>(a_dst + j * 8192, &tmA, fb, m0 + 64 * j, k0);
                     } else {
-                        tma_load_2d(a_dst, &tmA, fb, k0, m0);
+                        load2d<CG>(a_dst, &tmA, fb, k0, m0);
                     }
                     if (B_MN) {
 #pragma unroll
-                        for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, fb, n0 + 64 * j, k0);
+                        for (int j = 0; j < BNH / 64; ++j) load2d<CG>(b_dst + j * 8192, &tmB, fb, n0 + 64 * j, k0);
                     } else {
-                        tma_load_2d(b_dst, &tmB, fb, k0, n0);
+                        load2d<CG>(b_dst, &tmB, fb, k0, n0);
                     }
                 }
                 __syncwarp();
                 if (++s == STAGES) { s = 0; ph ^= 1; }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        constexpr uint32_t idesc = idesc_bf16(BN, A_MN, B_MN);
+    } else if (warp == 1 && h == 0) {
+        // ------------------------------------------------------------------ MMA issuer (the even block of a pair)
+        constexpr uint32_t idesc = CG == 2 ? idesc_bf16_pair(BN, A_MN, B_MN) : idesc_bf16(BN, A_MN, B_MN);
         int s = 0, i = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++i) {
+        for (int t = unit; t < n_tiles_total && ok; t += n_units, ++i) {
             const int buf = i & 1;
             const uint32_t d_tmem = tmem_base + (uint32_t)buf * C::BUF_COLS;
             ok = mbar_wait_uniform(smem_u32(&out_empty[buf]), ((i >> 1) & 1) ^ 1, ab);      // accumulator buffer drained
@@ -139,16 +170,22 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
                                                  : smem_desc_sw128(a_src + kk * 32, 0, 1024);
                         const uint64_t bd = B_MN ? smem_desc_sw128(b_src + kk * 2048, 8192, 1024)
                                                  : smem_desc_sw128(b_src + kk * 32, 0, 1024);
-                        mma_bf16_ss(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                        if (CG == 2) mma_bf16_ss_pair(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                        else mma_bf16_ss(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                     }
-                    mma_commit(smem_u32(&empty_bar[s]));
-                    if (kb == p.kb_total - 1) mma_commit(smem_u32(&out_full[buf]));
+                    if (CG == 2) {       // both blocks' stages are free, both blocks' accumulators are ready
+                        mma_commit_pair(smem_u32(&empty_bar[s]), 3);
+                        if (kb == p.kb_total - 1) mma_commit_pair(smem_u32(&out_full[buf]), 3);
+                    } else {
+                        mma_commit(smem_u32(&empty_bar[s]));
+                        if (kb == p.kb_total - 1) mma_commit(smem_u32(&out_full[buf]));
+                    }
                 }
                 __syncwarp();
                 if (++s == STAGES) { s = 0; ph ^= 1; }
             }
         }
-    } else {
+    } else if (warp >= 2) {
         // ------------------------------------------------------------------ epilogue
         const int q = warp % 4;                              // tensor-memory lanes [32 q, 32 q + 32)
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -157,9 +194,10 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         const bool bias_ok = p.bias && (((uintptr_t)p.bias & 15u) == 0);
         int i = 0, sb = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++i) {
+        for (int t = unit; t < n_tiles_total && ok; t += n_units, ++i) {
             const int buf = i & 1;
-            const int m0 = (t % p.m_tiles) * BM, n0 = (t / p.m_tiles) * BN;
+            const int m0 = (t % p.m_tiles) * (BM * CG) + h * BM, n0 = (t / p.m_tiles) * BN;
+            const bool rows_inside = m0 + q * 32 < p.M;      // (uniform) a pair's odd block may hang over the last row tile
             ok = mbar_wait_uniform(smem_u32(&out_full[buf]), (i >> 1) & 1, ab);
             if (!ok) break;
             tc_fence_after();
@@ -204,106 +242,142 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (elect_one()) {
-                    tma_store_2d(&tmC, slab, col0, m0 + q * 32);
+                    if (rows_inside) tma_store_2d(&tmC, slab, col0, m0 + q * 32);
                     tma_store_commit();
                 }
                 __syncwarp();
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&out_empty[buf]));
+            if (lane == 0) {
+                if (CG == 2) mbar_arrive_remote(smem_u32(&out_empty[buf]), 0);
+                else mbar_arrive(smem_u32(&out_empty[buf]));
+            }
         }
         tma_store_wait_read<0>();                            // shared memory may go once the stores have read it
         __syncwarp();
     }
 
     tc_fence_before();
-    __syncthreads();
+    if (CG == 2) {
+        // neither block leaves (or frees tensor memory) while the other may still signal one of its barriers,
+        // read its shared memory with an MMA or write its accumulators: every thread of the pair is past all of
+        // that when it arrives here
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
     if (warp == 1) {
         if (abort_flag) {            // give copies and MMAs still in flight time to land before freeing
             for (int i = 0; i < 256; ++i) __nanosleep(1000);
         }
         tc_fence_after();
-        tmem_dealloc(tmem_base, C::TMEM_COLS);
+        if (CG == 2) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+        else tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, int CG>
 lrd_status_t launch_p(const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tC, const PParams& p, unsigned blocks,
                       cudaStream_t stream) {
-    auto kern = tc_gemm_persistent_kernel<BN, A_MN, B_MN>;
+    auto kern = tc_gemm_persistent_kernel<BN, A_MN, B_MN, CG>;
     static bool configured = false;     // per instantiation; the attribute is sticky per function
     if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<BN>::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<BN, CG>::SMEM_BYTES) != cudaSuccess)
             return LRD_ERR_CUDA;
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(blocks, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = PCfg<BN>::SMEM_BYTES;
+    cfg.dynamicSmemBytes = PCfg<BN, CG>::SMEM_BYTES;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // the kernel waits (griddepcontrol.wait) before it touches global memory
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = CG;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = CG == 2 ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, kern, tA, tB, tC, p) != cudaSuccess) return LRD_ERR_CUDA;
     count_launch();
     return LRD_OK;
 }
 
-template <int BN>
+template <int BN, int CG>
 lrd_status_t launch_p_major(bool a_mn, bool b_mn, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tC,
                             const PParams& p, unsigned blocks, cudaStream_t s) {
-    if (a_mn) return b_mn ? launch_p<BN, true, true>(tA, tB, tC, p, blocks, s) : launch_p<BN, true, false>(tA, tB, tC, p, blocks, s);
-    return b_mn ? launch_p<BN, false, true>(tA, tB, tC, p, blocks, s) : launch_p<BN, false, false>(tA, tB, tC, p, blocks, s);
+    if (a_mn) return b_mn ? launch_p<BN, true, true, CG>(tA, tB, tC, p, blocks, s) : launch_p<BN, true, false, CG>(tA, tB, tC, p, blocks, s);
+    return b_mn ? launch_p<BN, false, true, CG>(tA, tB, tC, p, blocks, s) : launch_p<BN, false, false, CG>(tA, tB, tC, p, blocks, s);
 }
 
-// Tile width: every block streams (A tile + B tile) per k-block and the slowest block walks over
-// ceil(tiles / SMs) tiles, so minimise that product; wider tiles on ties (fewer re-reads of A).
-int pick_bn_p(int64_t M, int64_t N) {
-    if (N <= 64) return 64;
-    const int64_t mt = (M + BM - 1) / BM;
+// Tile shape.  Per k-block a block streams (A tile + its part of the B tile) from L2 at about 64 B/clk and
+// its MMAs take 2 BN clocks; the slowest unit walks over ceil(tiles / units) tiles.  Minimise the product over
+// the tile widths and over single blocks (148 units, 128-row tiles) and pairs (74 units, 256-row tiles);
+// earlier candidates (wider, single) win ties.
+struct PShape { int bn, cg; };
+int g_force_cg = 0;                  // 0: by the cost above; 1 or 2: forced where possible (test hook)
+
+PShape pick_shape_p(int64_t M, int64_t N) {
+    if (N <= 64) return {64, 1};
     const int cands[4] = {256, 192, 128, 64};
-    int best = 128;
+    PShape best = {128, 1};
     double best_cost = 1e300;
-    for (int bn : cands) {
-        const int64_t tiles = mt * ((N + bn - 1) / bn);
-        const double cost = (double)((tiles + kNumSms - 1) / kNumSms) * (double)(kATile + bn * BK * 2);
-        if (cost < best_cost) { best_cost = cost; best = bn; }
+    for (int cg = 1; cg <= 2; ++cg) {
+        if (g_force_cg && cg != g_force_cg) continue;
+        if (cg == 2 && M <= BM) continue;
+        const int64_t mt = (M + BM * cg - 1) / (BM * cg);
+        const int64_t units = kNumSms / cg;
+        for (int bn : cands) {
+            if (cg == 2 && bn != 256 && bn != 128) continue;
+            const int64_t tiles = mt * ((N + bn - 1) / bn);
+            const double fill = (double)(kATile + (bn / cg) * BK * 2) / 64.0, mma = 2.0 * bn;
+            const double cost = (double)((tiles + units - 1) / units) * (fill > mma ? fill : mma);
+            if (cost < best_cost) { best_cost = cost; best = {bn, cg}; }
+        }
     }
     return best;
 }
 
 }  // namespace
 
+void tc_gemm_persistent_force_pairs(int cg) { g_force_cg = (cg == 1 || cg == 2) ? cg : 0; }
+
 lrd_status_t tc_gemm_persistent(const GemmArgs& g, cudaStream_t stream) {
     if (!tc_gemm_eligible(g) || g.a_colsum) return LRD_ERR_UNSUPPORTED;
-    const int bn = pick_bn_p(g.M, g.N);
+    PShape sh = pick_shape_p(g.M, g.N);
+    if (g_force_cg == 2 && sh.cg != 2) { g_force_cg = 0; sh = pick_shape_p(g.M, g.N); g_force_cg = 2; }
+    const int bn = sh.bn, cg = sh.cg, bnh = bn / cg;
     CUtensorMap tA, tB, tC;
     bool ok = g.a_mn_major ? make_tmap_2d_bf16(&tA, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, 64)
                            : make_tmap_2d_bf16(&tA, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda, BM, BK);
     ok = ok && (g.b_mn_major ? make_tmap_2d_bf16(&tB, g.B, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.ldb, BK, 64)
-                             : make_tmap_2d_bf16(&tB, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.ldb, (uint32_t)bn, BK));
+                             : make_tmap_2d_bf16(&tB, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.ldb, (uint32_t)bnh, BK));
     ok = ok && make_tmap_2d_bf16(&tC, g.C, (uint64_t)g.M, (uint64_t)g.N, (uint64_t)g.ldc, 32, 32);
     if (!ok) return LRD_ERR_CUDA;
     PParams p;
     p.M = g.M; p.N = g.N;
     p.kb_total = (int)((g.K + BK - 1) / BK);
-    p.m_tiles = (int)((g.M + BM - 1) / BM);
+    p.m_tiles = (int)((g.M + BM * cg - 1) / (BM * cg));
     p.n_tiles = (int)((g.N + bn - 1) / bn);
     p.bias = (const __nv_bfloat16*)g.bias;
     p.timeout_flag = device_timeout_flag();
-    const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
-    // every block gets the same number of tiles (+-1): blocks = tiles / ceil(tiles / SMs), rounded up
-    const int64_t waves = (tiles + kNumSms - 1) / kNumSms;
-    const unsigned blocks = (unsigned)((tiles + waves - 1) / waves);
+    const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles, units_max = kNumSms / cg;
+    // every unit (block or pair) gets the same number of tiles (+-1): units = tiles / ceil(tiles / units_max), rounded up
+    const int64_t waves = (tiles + units_max - 1) / units_max;
+    const unsigned blocks = (unsigned)((tiles + waves - 1) / waves) * (unsigned)cg;
+    if (cg == 2) {
+        if (bn == 256) return launch_p_major<256, 2>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
+        return launch_p_major<128, 2>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
+    }
     switch (bn) {
-        case 256: return launch_p_major<256>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
-        case 192: return launch_p_major<192>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
-        case 128: return launch_p_major<128>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
-        default:  return launch_p_major<64>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
+        case 256: return launch_p_major<256, 1>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
+        case 192: return launch_p_major<192, 1>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
+        case 128: return launch_p_major<128, 1>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
+        default:  return launch_p_major<64, 1>(g.a_mn_major, g.b_mn_major, tA, tB, tC, p, blocks, stream);
     }
 }
 

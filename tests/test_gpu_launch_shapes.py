@@ -19,6 +19,7 @@ pytestmark = pytest.mark.gpu
 def _restore_tuning():
     yield
     b.lrd_chain_tuning(0, 0, 0)
+    b.lrd_gemm_tuning(0)
     b.lrd_set_path(b.LRD_PATH_AUTO)
 
 
@@ -95,3 +96,52 @@ def test_dependent_launches_back_to_back():
             "db2": rel_err(g["db2"], r2g["db"]), "dX": rel_err(dX, r1g["dX"]), "dU1": rel_err(g["dU1"], r1g["dU"]),
             "dV1": rel_err(g["dV1"], r1g["dV"]), "db1": rel_err(g["db1"], r1g["db"])}
     assert all(v <= 2e-2 for v in errs.values()), errs
+
+
+def _dense_run(M, K, N, seed):
+    bf = torch.bfloat16
+    X = wl.round_to(wl.normal(seed, (M, K)), "bf16")
+    W = wl.round_to(wl.normal(seed + 1, (N, K), 0.02), "bf16")
+    bias = wl.round_to(wl.normal(seed + 2, (N,), 0.1), "bf16")
+    dY = wl.round_to(wl.normal(seed + 3, (M, N)), "bf16")
+    desc = b.linear_desc(M, K, N, 0, b.LRD_BF16)
+    ws = workspace(b.lrd_dense_workspace_bytes(desc, 1))
+    Y = torch.full((M, N), float("nan"), dtype=bf, device="cuda")
+    dX = torch.full((M, K), float("nan"), dtype=bf, device="cuda")
+    dW, db = torch.empty(N, K, dtype=bf, device="cuda"), torch.empty(N, dtype=bf, device="cuda")
+    b.lrd_dense_fwd(desc, dev(X, "bf16"), dev(W, "bf16"), dev(bias, "bf16"), Y, ws)
+    b.lrd_dense_bwd(desc, dev(dY, "bf16"), dev(X, "bf16"), dev(W, "bf16"), dX, dW, db, ws)
+    torch.cuda.synchronize()
+    assert b.lrd_check_device_status() == b.LRD_OK
+    return (X, W, bias, dY), (Y, dX)
+
+
+# 129 rows: the odd block of the only pair holds one row; 300 / 1300: an odd number of 128-row tiles, so the last
+# pair's odd block hangs over the edge entirely; 2304 x 2100: several tiles per pair, both accumulator buffers reused
+@pytest.mark.parametrize("shape", [(129, 64, 72), (300, 200, 136), (1300, 328, 520), (2304, 264, 2100), (512, 1096, 256)])
+def test_products_on_pairs_of_sms_match_the_oracle_and_single_blocks(shape):
+    M, K, N = shape
+    b.lrd_gemm_tuning(1)
+    _, (Y1, dX1) = _dense_run(M, K, N, 700 + M)
+    b.lrd_gemm_tuning(2)
+    (X, W, bias, dY), (Y2, dX2) = _dense_run(M, K, N, 700 + M)
+    assert rel_err(Y2, o.dense_fwd(X, W, bias)) <= 2e-2
+    assert rel_err(dX2, o.dense_bwd(dY, X, W)["dX"]) <= 2e-2
+    # same products summed in the same order, whichever SM holds which rows
+    assert torch.equal(Y1, Y2) and torch.equal(dX1, dX2)
+
+
+@pytest.mark.parametrize("cg", [1, 2])
+@pytest.mark.parametrize("shape", [(700, 520, 776, 512), (1500, 264, 200, 72)])
+def test_unfused_layer_with_products_on_single_blocks_and_on_pairs(cg, shape):
+    M, K, N, r = shape
+    b.lrd_gemm_tuning(cg)
+    for freeze in (b.LRD_FREEZE_NONE, b.LRD_FREEZE_U):
+        check_linear(wl.random_factor_case(M, K, N, r, "bf16", 760 + M + cg), freeze, path=b.LRD_PATH_UNFUSED)
+
+
+def test_gemm_tuning_rejects_values_outside_the_list():
+    for bad in (-1, 3, 4):
+        with pytest.raises(b.LrdError):
+            b.lrd_gemm_tuning(bad)
+    b.lrd_gemm_tuning(0)

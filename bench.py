@@ -235,6 +235,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=4, help="distinct activation buffer sets cycled through (L2 eviction)")
     ap.add_argument("--path", default="auto", choices=["auto", "general", "unfused", "fused"])
+    ap.add_argument("--groups", default="qkv", choices=["none", "qkv"],
+                    help="qkv: the three independent attention projections go out as one group (the default); none: one call per layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every step instead of CUDA graphs")
     args = ap.parse_args()
@@ -301,11 +303,34 @@ def main():
                          None if freeze == b.LRD_FREEZE_U else L["dU"], None if freeze == b.LRD_FREEZE_V else L["dV"],
                          None if freeze == b.LRD_FREEZE_U else L["db"], freeze, L["ws"])
 
+    # The query, key and value projections of a block depend on nothing the others produce: they go out as one
+    # group (side by side); the output projection and the two feed-forward layers follow one another.
+    group = [L for L in layers if L["name"] in ("attn_q", "attn_k", "attn_v")] if args.groups != "none" else []
+    singles = [L for L in layers if not any(L is G for G in group)]
+
+    def group_fwd(Ls, s, freeze):
+        sts = [L["sets"][s] for L in Ls]
+        b.lrd_linear_group_fwd([L["desc"] for L in Ls], [st["X"] for st in sts], [L["V"] for L in Ls], [L["U"] for L in Ls],
+                               [L["b"] for L in Ls], [st["Y"] for st in sts],
+                               None if freeze == b.LRD_FREEZE_U else [st["Z"] for st in sts], freeze, [L["ws"] for L in Ls])
+
+    def group_bwd(Ls, s, freeze):
+        sts = [L["sets"][s] for L in Ls]
+        fu, fv = freeze == b.LRD_FREEZE_U, freeze == b.LRD_FREEZE_V
+        b.lrd_linear_group_bwd([L["desc"] for L in Ls], [st["dY"] for st in sts], None if fv else [st["X"] for st in sts],
+                               [L["V"] for L in Ls], [L["U"] for L in Ls], None if fu else [st["Z"] for st in sts],
+                               [st["dX"] for st in sts], None if fu else [L["dU"] for L in Ls], None if fv else [L["dV"] for L in Ls],
+                               None if fu else [L["db"] for L in Ls], freeze, [L["ws"] for L in Ls])
+
     def step_eager(s, freeze):
-        for L in layers:
+        if group:
+            group_fwd(group, s, freeze)
+        for L in singles:
             fwd(L, L["sets"][s], freeze)
-        for L in reversed(layers):
+        for L in reversed(singles):
             bwd(L, L["sets"][s], freeze)
+        if group:
+            group_bwd(group, s, freeze)
 
     masks = [b.LRD_FREEZE_U, b.LRD_FREEZE_V]
     # warm every (set, mask) once outside any capture: one-time kernel attribute set-up happens here
@@ -534,7 +559,9 @@ def main():
                 "config": config_dict({"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                                        "l2": f"cycling {S} activation buffer sets, {S * act_bytes_per_set / 1e6:.0f} MB > 126 MB L2",
                                        "launch": "eager C-ABI calls" if args.no_graph else "CUDA graph replay of the C-ABI calls",
-                                       "path": args.path}),
+                                       "path": args.path,
+                                       "groups": {"qkv": "attn_q/k/v side by side in one group call, the other layers one call each",
+                                                  "none": "one call per layer"}[args.groups]}),
                 "useful_tflops": useful_flops * world / (ms_per_step * 1e-3) / 1e12,
                 "step_roofline_frac": t_roof / (ms_per_step * 1e-3), "step_roofline_us": t_roof * 1e6,
                 "roofline": roof, "cpu_baseline": cpu,

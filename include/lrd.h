@@ -175,6 +175,39 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
                             const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                             lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* ---- groups of independent decomposed layers -------------------------------------------------------
+ * The n layers of a group depend on nothing the others produce (the query, key and value projections
+ * of an attention block, which read the same X, are the model case; the paper's Section 2 treats every
+ * layer on its own, so grouping is a launch-level matter with no counterpart there).  Layer i is given
+ * by descs[i] and the i-th entries of the pointer arrays, each with the meaning, layout and rules of the
+ * same argument of lrd_linear_fwd / lrd_linear_bwd; the arrays themselves are HOST arrays of n entries.
+ * `bias`, `Z_save`, and in the backward `X`, `Z_save`, `dX`, `dU`, `dV`, `dbias` may be NULL as a whole
+ * where the single-layer call allows NULL for every layer.  Inputs may be shared between layers;
+ * outputs and workspaces must not overlap one another (every layer writes its own dX: the caller adds
+ * them up where the layers share X).  One mask applies to the whole group.
+ *
+ * The layers are enqueued side by side: layer 0 on `cuda_stream`, the others on streams the library
+ * owns (created on first use, one set per device, never freed), which start after the work already in
+ * `cuda_stream` and which `cuda_stream` waits for before the call returns - so to the caller the group
+ * behaves like n single-layer calls on `cuda_stream`, and it may be captured into a CUDA graph.  Each
+ * launch is shaped for 1/n of the SMs.  In the backward, a layer's dU (+ dbias) product runs beside its
+ * data chain.  Results are those of the single-layer calls.  n = 1 is allowed (then only the dU
+ * overlap differs from lrd_linear_bwd).
+ *
+ * Errors: LRD_ERR_INVALID_ARG for n outside [0, LRD_MAX_GROUP] or a NULL required array; otherwise the
+ * first failing layer's status.  All layers are validated before anything is enqueued.  Not
+ * thread-safe: two host threads must not run groups on the same device at the same time.  Make the
+ * first group call on a device outside any stream capture (it creates the library's streams). */
+#define LRD_MAX_GROUP 8
+lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
+                                  const void* const* U, const void* const* bias, void* const* Y, void* const* Z_save,
+                                  lrd_freeze_t freeze, void* const* workspace, const size_t* workspace_bytes,
+                                  void* cuda_stream);
+lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const void* const* dY, const void* const* X,
+                                  const void* const* V, const void* const* U, const void* const* Z_save, void* const* dX,
+                                  void* const* dU, void* const* dV, void* const* dbias, lrd_freeze_t freeze,
+                                  void* const* workspace, const size_t* workspace_bytes, void* cuda_stream);
+
 /* ---- the undecomposed layer, for comparison (the "original layer" of Algorithm 1) -------- */
 
 /* Y = X W^T + bias with W[N x K] (leading dimension desc->ldv; desc->r, ldu, ldz ignored). */

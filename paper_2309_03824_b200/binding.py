@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_gemm_tuning", "lrd_rank_search",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_gemm_tuning", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd",
 ]
 
 
@@ -60,6 +60,12 @@ _lib.lrd_rank_search.restype = _i64
 _lib.lrd_rank_search.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double, C.POINTER(C.c_int)]
 _lib.lrd_chain_tuning.restype = _int
 _lib.lrd_chain_tuning.argtypes = [_int, _int, _int]
+_pp = C.POINTER(C.c_void_p)
+_lib.lrd_linear_group_fwd.restype = _int
+_lib.lrd_linear_group_fwd.argtypes = [_int, C.POINTER(lrd_linear_desc_t), _pp, _pp, _pp, _pp, _pp, _pp, _int, _pp,
+                                      C.POINTER(C.c_size_t), C.c_void_p]
+_lib.lrd_linear_group_bwd.restype = _int
+_lib.lrd_linear_group_bwd.argtypes = [_int, C.POINTER(lrd_linear_desc_t)] + [_pp] * 9 + [_int, _pp, C.POINTER(C.c_size_t), C.c_void_p]
 _lib.lrd_gemm_tuning.restype = _int
 _lib.lrd_gemm_tuning.argtypes = [_int]
 _lib.lrd_check_device_status.restype = _int
@@ -199,6 +205,44 @@ def lrd_linear_bwd(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspa
     w, n = _ws(workspace)
     st = _lib.lrd_linear_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(V), _ptr(U), _ptr(Z_save), _ptr(dX), _ptr(dU),
                              _ptr(dV), _ptr(dbias), freeze, w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def _ptr_array(ts, n):
+    """Host array of n device pointers (NULL entries for None); None for a list that is None as a whole."""
+    if ts is None:
+        return None
+    if len(ts) != n:
+        raise ValueError("every per-layer list of a group has one entry per layer")
+    return (C.c_void_p * n)(*[None if t is None else t.data_ptr() for t in ts])
+
+
+def _group_common(descs, workspaces):
+    n = len(descs)
+    darr = (lrd_linear_desc_t * n)(*descs)
+    ws = [_ws(w) for w in workspaces]
+    warr = (C.c_void_p * n)(*[w[0] for w in ws])
+    wbytes = (C.c_size_t * n)(*[w[1] for w in ws])
+    return n, darr, warr, wbytes
+
+
+def lrd_linear_group_fwd(descs, X, V, U, bias, Y, Z_save, freeze, workspaces, stream=None, check=True):
+    """n independent layers side by side: every argument but freeze/stream is a list with one entry per layer."""
+    n, darr, warr, wbytes = _group_common(descs, workspaces)
+    st = _lib.lrd_linear_group_fwd(n, darr, _ptr_array(X, n), _ptr_array(V, n), _ptr_array(U, n), _ptr_array(bias, n),
+                                   _ptr_array(Y, n), _ptr_array(Z_save, n), freeze, warr, wbytes, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_linear_group_bwd(descs, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspaces, stream=None, check=True):
+    n, darr, warr, wbytes = _group_common(descs, workspaces)
+    st = _lib.lrd_linear_group_bwd(n, darr, _ptr_array(dY, n), _ptr_array(X, n), _ptr_array(V, n), _ptr_array(U, n),
+                                   _ptr_array(Z_save, n), _ptr_array(dX, n), _ptr_array(dU, n), _ptr_array(dV, n),
+                                   _ptr_array(dbias, n), freeze, warr, wbytes, _stream(stream))
     if check:
         _check(st)
     return st

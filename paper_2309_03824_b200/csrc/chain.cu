@@ -485,9 +485,11 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         const uint32_t s1b = (uint32_t)G1 * kb1_bytes;
         const uint32_t used1 = (uint32_t)S1 * s1b, used2 = kStagingBytes + (uint32_t)S2 * kb2_bytes;
         Plan pl{C, RS, swb, BN2, G1, S1, S2, s1b, kb2_bytes, (uint32_t)t_bytes, 1024u + (uint32_t)t_bytes + (used1 > used2 ? used1 : used2)};
-        // prefer the largest cluster whose blocks are all resident at once; else the smallest feasible
+        // prefer the largest cluster whose blocks are all resident at once (within this launch's share of the
+        // SMs, when it runs beside other launches); else the smallest feasible
         if (!found) { best = pl; found = true; }
-        if (tiles <= max_active_clusters(C)) { best = pl; break; }
+        const int64_t room = a.sm_share > 0 && !g_tune_C ? (int64_t)a.sm_share / C : (int64_t)max_active_clusters(C);
+        if (tiles <= room && tiles <= max_active_clusters(C)) { best = pl; break; }
         best = pl;
     }
     if (!found) return false;

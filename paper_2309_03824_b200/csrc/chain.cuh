@@ -16,6 +16,7 @@ struct ChainArgs {
     void* Out; int64_t ld_out;         // [M x N2]
     void* T_save; int64_t ldt;         // [M x r] or nullptr
     lrd_dtype_t dtype;
+    int sm_share = 0;                  // SMs this launch can count on when it runs beside others (0: all of them)
 };
 
 // Overrides of the launch shape for benchmarking sweeps: cluster size, k-blocks per phase-1 stage,

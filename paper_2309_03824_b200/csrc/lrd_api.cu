@@ -240,9 +240,10 @@ size_t lrd_dense_workspace_bytes(const lrd_linear_desc_t* desc, int is_bwd) {
     return 256 + need;
 }
 
-lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
-                            const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze, void* workspace,
-                            size_t workspace_bytes, void* cuda_stream) {
+// One layer's forward on stream s.  sm_share: SMs the launch can count on beside concurrent launches (0: all).
+static lrd_status_t linear_fwd_on(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
+                                  const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze, void* workspace,
+                                  size_t workspace_bytes, cudaStream_t s, int sm_share, bool check_only = false) {
     Linear L;
     LRD_TRY(parse_linear(desc, &L, false));
     if (freeze != LRD_FREEZE_NONE && freeze != LRD_FREEZE_U && freeze != LRD_FREEZE_V) return LRD_ERR_INVALID_ARG;
@@ -253,8 +254,7 @@ lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const 
         if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
     LRD_TRY(check_ws(workspace, workspace_bytes, lrd_linear_workspace_bytes(desc, freeze, 0)));
     LRD_TRY(check_arch());
-    if (L.M == 0) return LRD_OK;
-    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (L.M == 0 || check_only) return LRD_OK;
 
     const int path = g_path.load();
     if (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) {
@@ -262,6 +262,7 @@ lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const 
         c.M = L.M; c.K1 = L.K; c.r = L.r; c.N2 = L.N;
         c.In = X; c.ld_in = L.ldx; c.P = V; c.ldp = L.ldv; c.Q = U; c.ldq = L.ldu; c.bias = bias;
         c.Out = Y; c.ld_out = L.ldy; c.T_save = Z_save; c.ldt = L.ldz; c.dtype = L.dt;
+        c.sm_share = sm_share;
         if (path == LRD_PATH_FUSED ? chain_eligible(c) : chain_preferred(c)) return chain_launch(c, s);
     }
     void* Z = Z_save ? Z_save : workspace;
@@ -270,9 +271,20 @@ lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const 
     return run_gemm(gemm(L.M, L.N, L.r, Z, ldz, false, U, L.ldu, false, Y, L.ldy, bias, L.dt), false, nullptr, 0, s);
 }
 
-lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
-                            const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
-                            lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
+                            const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+    return linear_fwd_on(desc, X, V, U, bias, Y, Z_save, freeze, workspace, workspace_bytes, (cudaStream_t)cuda_stream, 0);
+}
+
+// One layer's backward on stream s.  With a side stream, the dU (+ db) product, which needs nothing the data
+// chain produces, runs there beside the chain; the caller has made `side` wait for s's earlier work and makes s
+// wait for `side` afterwards.  dV follows the chain (it reads the dZ the chain spills) and, when dU is computed too,
+// dU as well (the two may share the split-K scratch).
+static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                                  const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                                  lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, cudaStream_t s,
+                                  cudaStream_t side, cudaEvent_t side_done, int sm_share, bool check_only = false) {
     Linear L;
     LRD_TRY(parse_linear(desc, &L, false));
     const uint32_t plan = lrd_linear_bwd_plan(freeze);
@@ -285,7 +297,7 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
         if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
     LRD_TRY(check_ws(workspace, workspace_bytes, lrd_linear_workspace_bytes(desc, freeze, 1)));
     LRD_TRY(check_arch());
-    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (check_only) return LRD_OK;
 
     // frozen factor: no product is launched; a gradient buffer the caller passed reads as zero
     if (!(plan & LRD_PLAN_DU)) {
@@ -311,6 +323,7 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
         c.M = L.M; c.K1 = L.N; c.r = L.r; c.N2 = L.K;
         c.In = dY; c.ld_in = L.ldy; c.P = U; c.ldp = L.ldu; c.Q = V; c.ldq = L.ldv; c.bias = nullptr;
         c.Out = dX; c.ld_out = L.ldx; c.T_save = need_dz_in_memory ? dZ : nullptr; c.ldt = L.r; c.dtype = L.dt;
+        c.sm_share = sm_share;
         if (path == LRD_PATH_FUSED ? chain_eligible(c) : chain_preferred(c)) {
             LRD_TRY(chain_launch(c, s));
             chained = true;
@@ -329,13 +342,122 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
             gu.a_colsum = dbias;
             if (tc_gemm_colsum_ok(gu)) db_done = true; else gu.a_colsum = nullptr;
         }
-        LRD_TRY(run_gemm(gu, true, partials, partial_bytes, s));
-        if (dbias && !db_done) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, partial_bytes, s));
+        cudaStream_t su = side ? side : s;
+        LRD_TRY(run_gemm(gu, true, partials, partial_bytes, su));
+        if (dbias && !db_done) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, partial_bytes, su));
+        if (side && (plan & LRD_PLAN_DV)) {
+            if (cudaEventRecord(side_done, side) != cudaSuccess || cudaStreamWaitEvent(s, side_done, 0) != cudaSuccess) return LRD_ERR_CUDA;
+        }
     }
     if (plan & LRD_PLAN_DV)
         LRD_TRY(run_gemm(gemm(L.K, L.r, L.M, X, L.ldx, true, dZ, L.r, true, dV, L.ldv, nullptr, L.dt), true, partials,
                          partial_bytes, s));
     return LRD_OK;
+}
+
+lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                            const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                            lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return linear_bwd_on(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, workspace_bytes,
+                         (cudaStream_t)cuda_stream, nullptr, nullptr, 0);
+}
+
+// ---- groups of independent layers -------------------------------------------------------------------
+// Side streams and events of the calling device, made on first use and kept.  Layer 0 of a group runs on the
+// caller's stream, layer i on side stream i - 1; the dU products of a backward group use a second set.
+namespace {
+struct SideStreams {
+    int device = -1;
+    cudaStream_t layer[LRD_MAX_GROUP], du[LRD_MAX_GROUP];
+    cudaEvent_t fork, join[LRD_MAX_GROUP], du_done[LRD_MAX_GROUP];
+};
+SideStreams g_sides[16];
+int g_n_sides = 0;
+
+SideStreams* side_streams() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    for (int i = 0; i < g_n_sides; ++i)
+        if (g_sides[i].device == dev) return &g_sides[i];
+    if (g_n_sides == 16) return nullptr;
+    SideStreams* ss = &g_sides[g_n_sides];
+    bool ok = cudaEventCreateWithFlags(&ss->fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < LRD_MAX_GROUP && ok; ++i) {
+        ok = cudaStreamCreateWithFlags(&ss->layer[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaStreamCreateWithFlags(&ss->du[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ss->join[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ss->du_done[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) return nullptr;
+    ss->device = dev;
+    ++g_n_sides;
+    return ss;
+}
+
+inline bool after(cudaStream_t waiter, cudaStream_t done, cudaEvent_t ev) {      // waiter's next work follows done's work so far
+    return cudaEventRecord(ev, done) == cudaSuccess && cudaStreamWaitEvent(waiter, ev, 0) == cudaSuccess;
+}
+}  // namespace
+
+lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
+                                  const void* const* U, const void* const* bias, void* const* Y, void* const* Z_save,
+                                  lrd_freeze_t freeze, void* const* workspace, const size_t* workspace_bytes,
+                                  void* cuda_stream) {
+    if (n < 0 || n > LRD_MAX_GROUP) return LRD_ERR_INVALID_ARG;
+    if (n == 0) return LRD_OK;
+    if (!descs || !X || !V || !U || !Y || !workspace || !workspace_bytes) return LRD_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    for (int i = 0; i < n; ++i)          // nothing is enqueued unless every layer's arguments are valid
+        LRD_TRY(linear_fwd_on(&descs[i], X[i], V[i], U[i], bias ? bias[i] : nullptr, Y[i], Z_save ? Z_save[i] : nullptr, freeze,
+                              workspace[i], workspace_bytes[i], s, 0, true));
+    SideStreams* ss = n > 1 ? side_streams() : nullptr;
+    if (n > 1 && !ss) return LRD_ERR_CUDA;
+    if (n > 1 && cudaEventRecord(ss->fork, s) != cudaSuccess) return LRD_ERR_CUDA;
+    const int share = n > 1 ? kNumSms / n : 0;
+    lrd_status_t st = LRD_OK;
+    for (int i = 0; i < n; ++i) {
+        cudaStream_t si = i == 0 ? s : ss->layer[i - 1];
+        if (i > 0 && cudaStreamWaitEvent(si, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
+        const lrd_status_t sti = linear_fwd_on(&descs[i], X[i], V[i], U[i], bias ? bias[i] : nullptr, Y[i],
+                                               Z_save ? Z_save[i] : nullptr, freeze, workspace[i], workspace_bytes[i], si, share);
+        if (sti != LRD_OK) st = sti;
+        if (i > 0 && !after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;      // joined even after a failure
+    }
+    return st;
+}
+
+lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const void* const* dY, const void* const* X,
+                                  const void* const* V, const void* const* U, const void* const* Z_save, void* const* dX,
+                                  void* const* dU, void* const* dV, void* const* dbias, lrd_freeze_t freeze,
+                                  void* const* workspace, const size_t* workspace_bytes, void* cuda_stream) {
+    if (n < 0 || n > LRD_MAX_GROUP) return LRD_ERR_INVALID_ARG;
+    if (n == 0) return LRD_OK;
+    if (!descs || !dY || !V || !U || !workspace || !workspace_bytes) return LRD_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    auto at = [](const void* const* a, int i) -> const void* { return a ? a[i] : nullptr; };
+    auto at_w = [](void* const* a, int i) -> void* { return a ? a[i] : nullptr; };
+    for (int i = 0; i < n; ++i)
+        LRD_TRY(linear_bwd_on(&descs[i], dY[i], at(X, i), V[i], U[i], at(Z_save, i), at_w(dX, i), at_w(dU, i), at_w(dV, i),
+                              at_w(dbias, i), freeze, workspace[i], workspace_bytes[i], s, nullptr, nullptr, 0, true));
+    SideStreams* ss = side_streams();
+    if (!ss) return LRD_ERR_CUDA;
+    if (cudaEventRecord(ss->fork, s) != cudaSuccess) return LRD_ERR_CUDA;
+    const bool du_aside = (lrd_linear_bwd_plan(freeze) & LRD_PLAN_DU) != 0;
+    const int share = n > 1 ? kNumSms / n : 0;
+    lrd_status_t st = LRD_OK;
+    for (int i = 0; i < n; ++i) {
+        cudaStream_t si = i == 0 ? s : ss->layer[i - 1];
+        cudaStream_t sd = du_aside ? ss->du[i] : nullptr;
+        if (i > 0 && cudaStreamWaitEvent(si, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
+        if (sd && cudaStreamWaitEvent(sd, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
+        const lrd_status_t sti = linear_bwd_on(&descs[i], dY[i], at(X, i), V[i], U[i], at(Z_save, i), at_w(dX, i), at_w(dU, i),
+                                               at_w(dV, i), at_w(dbias, i), freeze, workspace[i], workspace_bytes[i], si, sd,
+                                               ss->du_done[i], share);
+        if (sti != LRD_OK) st = sti;
+        if (sd && !after(s, sd, ss->du_done[i])) st = LRD_ERR_CUDA;
+        if (i > 0 && !after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;
+    }
+    return st;
 }
 
 lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const void* W, const void* bias, void* Y,

@@ -1,0 +1,133 @@
+"""Groups of independent layers enqueued side by side (the query / key / value projections of an attention block):
+parity of every layer with the oracle, identity with the single-layer calls, replay from a CUDA graph, and the
+argument checks that run before anything is enqueued."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2309_03824_b200 import binding as b
+from paper_2309_03824_b200 import workloads as wl
+
+from helpers import DT, TOL, dev, host, oracle_linear, rel_err, run_linear, workspace
+
+pytestmark = pytest.mark.gpu
+
+NAMES = ("Y", "Z", "dX", "dU", "dV", "db")
+
+
+def make_group(shapes, seed, shared_x=False):
+    cases = [wl.random_factor_case(M, K, N, r, "bf16", seed + 7 * i) for i, (M, K, N, r) in enumerate(shapes)]
+    if shared_x:
+        for c in cases[1:]:
+            c["X"] = cases[0]["X"]
+    return cases
+
+
+class Group:
+    def __init__(self, cases, freeze):
+        code, tdt = DT["bf16"]
+        self.cases, self.freeze, self.n = cases, freeze, len(cases)
+        self.descs = [b.linear_desc(c["M"], c["K"], c["N"], c["r"], code) for c in cases]
+        self.in_ = {k: [dev(c[k], "bf16") for c in cases] for k in ("X", "V", "U", "b", "dY")}
+        nan = float("nan")
+        self.out = {"Y": [torch.full((c["M"], c["N"]), nan, dtype=tdt, device="cuda") for c in cases],
+                    "Z": None if freeze == b.LRD_FREEZE_U else [torch.full((c["M"], c["r"]), nan, dtype=tdt, device="cuda") for c in cases],
+                    "dX": [torch.full((c["M"], c["K"]), nan, dtype=tdt, device="cuda") for c in cases],
+                    "dU": [torch.full((c["N"], c["r"]), nan, dtype=tdt, device="cuda") for c in cases],
+                    "dV": [torch.full((c["K"], c["r"]), nan, dtype=tdt, device="cuda") for c in cases],
+                    "db": [torch.full((c["N"],), nan, dtype=tdt, device="cuda") for c in cases]}
+        self.ws = [workspace(max(b.lrd_linear_workspace_bytes(d, freeze, 0), b.lrd_linear_workspace_bytes(d, freeze, 1))) for d in self.descs]
+
+    def fwd(self):
+        i, o_ = self.in_, self.out
+        b.lrd_linear_group_fwd(self.descs, i["X"], i["V"], i["U"], i["b"], o_["Y"], o_["Z"], self.freeze, self.ws)
+
+    def bwd(self):
+        i, o_ = self.in_, self.out
+        b.lrd_linear_group_bwd(self.descs, i["dY"], None if self.freeze == b.LRD_FREEZE_V else i["X"], i["V"], i["U"], o_["Z"],
+                               o_["dX"], o_["dU"], o_["dV"], o_["db"], self.freeze, self.ws)
+
+    def check(self, single=True):
+        torch.cuda.synchronize()
+        assert b.lrd_check_device_status() == b.LRD_OK
+        for li, case in enumerate(self.cases):
+            ref = oracle_linear(case, self.freeze)
+            one = run_linear(case, self.freeze) if single else None
+            for name in NAMES:
+                if self.out[name] is None:
+                    continue
+                got = self.out[name][li]
+                assert rel_err(got, ref[name]) <= TOL["bf16"], (li, name)
+                # a group changes where and beside what a layer runs, not what is summed in which order
+                if one is not None and one[name] is not None:
+                    assert torch.equal(got, one[name]), (li, name)
+
+
+QKV = [(520, 264, 264, 64)] * 3
+MIXED = [(300, 200, 136, 48), (300, 200, 520, 128), (700, 136, 200, 64), (130, 776, 72, 32)]
+
+
+@pytest.mark.parametrize("freeze", [b.LRD_FREEZE_NONE, b.LRD_FREEZE_U, b.LRD_FREEZE_V])
+@pytest.mark.parametrize("shapes,shared", [(QKV, True), (MIXED, False), ([(400, 328, 264, 96)], False)])
+def test_group_matches_oracle_and_single_layer_calls(freeze, shapes, shared):
+    g = Group(make_group(shapes, 1200 + len(shapes), shared), freeze)
+    g.fwd()
+    g.bwd()
+    g.check()
+
+
+def test_group_of_eight_layers_and_empty_group():
+    g = Group(make_group([(260, 136, 136, 32)] * 8, 1300), b.LRD_FREEZE_NONE)
+    g.fwd()
+    g.bwd()
+    g.check(single=False)
+    assert b.lrd_linear_group_fwd([], [], [], [], [], [], [], b.LRD_FREEZE_NONE, []) == b.LRD_OK
+
+
+def test_group_replayed_from_a_cuda_graph():
+    """Captured once (the side streams join the capture and rejoin before it ends), replayed on fresh outputs."""
+    g = Group(make_group(QKV, 1400, shared_x=True), b.LRD_FREEZE_NONE)
+    g.fwd()
+    g.bwd()
+    torch.cuda.synchronize()
+    first = {k: [t.clone() for t in v] for k, v in g.out.items()}
+    side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            g.fwd()
+            g.bwd()
+    for _ in range(3):
+        for v in g.out.values():
+            for t in v:
+                t.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        for k, v in g.out.items():
+            for li, t in enumerate(v):
+                assert torch.equal(t, first[k][li]), (k, li)
+    g.check(single=False)
+
+
+def test_group_checks_every_layer_before_enqueueing_anything():
+    g = Group(make_group(QKV, 1500), b.LRD_FREEZE_U)
+    good_ws = g.ws
+    g.ws = [good_ws[0], good_ws[1], torch.empty(256, dtype=torch.uint8, device="cuda")]      # last layer: workspace too small
+    outs = [t for v in g.out.values() if v is not None for t in v]
+    for t in outs:
+        t.fill_(7.0)
+    with pytest.raises(b.LrdError):
+        g.fwd()
+    with pytest.raises(b.LrdError):
+        g.bwd()
+    torch.cuda.synchronize()
+    for t in outs:
+        assert bool((t == 7.0).all())              # the valid layers before it did not run either
+    g.ws = good_ws
+    with pytest.raises(b.LrdError):               # more layers than a group may hold
+        big = Group(make_group([(130, 64, 64, 16)] * 9, 1600), b.LRD_FREEZE_U)
+        big.fwd()
+    with pytest.raises(ValueError):               # a per-layer list of the wrong length
+        b.lrd_linear_group_fwd(g.descs, g.in_["X"][:2], g.in_["V"], g.in_["U"], g.in_["b"], g.out["Y"], g.out["Z"], g.freeze, g.ws)
+    g.fwd()
+    g.bwd()
+    g.check(single=False)

@@ -443,7 +443,10 @@ lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const v
     if (!ss) return LRD_ERR_CUDA;
     if (cudaEventRecord(ss->fork, s) != cudaSuccess) return LRD_ERR_CUDA;
     const bool du_aside = (lrd_linear_bwd_plan(freeze) & LRD_PLAN_DU) != 0;
-    const int share = n > 1 ? kNumSms / n : 0;
+    // The data chains are shaped for twice their even share: the weight-gradient launches that follow each of them
+    // fill the machine anyway, and a chain of 2 blocks per row tile finishes sooner than one of 1 (three
+    // 768 -> 768, r = 192 layers at 4096 tokens, U frozen: 32.9 us against 35.3 us).
+    const int share = n > 1 ? 2 * kNumSms / n : 0;
     lrd_status_t st = LRD_OK;
     for (int i = 0; i < n; ++i) {
         cudaStream_t si = i == 0 ? s : ss->layer[i - 1];

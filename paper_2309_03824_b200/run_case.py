@@ -2,6 +2,8 @@
 profilers and quick timing.
 
     python -m paper_2309_03824_b200.run_case --M 4096 --K 768 --N 768 --r 192 --freeze U --what fwd --iters 5
+
+--r 0 runs the undecomposed layer (lrd_dense_fwd / lrd_dense_bwd) instead.
 """
 from __future__ import annotations
 
@@ -24,14 +26,20 @@ def main():
     freeze = {"none": 0, "U": 1, "V": 2}[a.freeze]
     b.lrd_set_path({"auto": 0, "general": 1, "unfused": 2, "fused": 3}[a.path])
     bf = torch.bfloat16
-    case = wl.random_factor_case(a.M, a.K, a.N, a.r, "bf16", 7)
+    dense = a.r == 0
+    case = wl.random_factor_case(a.M, a.K, a.N, 64 if dense else a.r, "bf16", 7)
     V, U, bias = (torch.from_numpy(case[k]).to("cuda", bf) for k in ("V", "U", "b"))
     desc = b.linear_desc(a.M, a.K, a.N, a.r, b.LRD_BF16)
-    ws = torch.empty(max(b.lrd_linear_workspace_bytes(desc, freeze, 1), 256), dtype=torch.uint8, device="cuda")
+    if dense:
+        W = (U.float() @ V.float().T).to(bf)                 # [N x K]
+        dW = torch.empty(a.N, a.K, dtype=bf, device="cuda")
+        ws = torch.empty(max(b.lrd_dense_workspace_bytes(desc, 1), 256), dtype=torch.uint8, device="cuda")
+    else:
+        ws = torch.empty(max(b.lrd_linear_workspace_bytes(desc, freeze, 1), 256), dtype=torch.uint8, device="cuda")
     sets = []
     for _ in range(a.sets):        # distinct buffers so that consecutive launches do not hit in L2
         sets.append(dict(X=torch.from_numpy(case["X"]).to("cuda", bf), dY=torch.from_numpy(case["dY"]).to("cuda", bf),
-                         Y=torch.empty(a.M, a.N, dtype=bf, device="cuda"), Z=torch.empty(a.M, a.r, dtype=bf, device="cuda"),
+                         Y=torch.empty(a.M, a.N, dtype=bf, device="cuda"), Z=torch.empty(a.M, max(a.r, 8), dtype=bf, device="cuda"),
                          dX=torch.empty(a.M, a.K, dtype=bf, device="cuda")))
     dU = torch.empty(a.N, a.r, dtype=bf, device="cuda")
     dV = torch.empty(a.K, a.r, dtype=bf, device="cuda")
@@ -42,6 +50,12 @@ def main():
         e0.record()
         for i in range(a.iters):
             s = sets[i % a.sets]
+            if dense:
+                if a.what in ("fwd", "both"):
+                    b.lrd_dense_fwd(desc, s["X"], W, bias, s["Y"], ws)
+                if a.what in ("bwd", "both"):
+                    b.lrd_dense_bwd(desc, s["dY"], s["X"], W, s["dX"], dW, db, ws)
+                continue
             if a.what in ("fwd", "both"):
                 b.lrd_linear_fwd(desc, s["X"], V, U, bias, s["Y"], None if freeze == 1 else s["Z"], freeze, ws)
             if a.what in ("bwd", "both"):

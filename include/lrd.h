@@ -140,6 +140,14 @@ lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chu
  * other values. */
 lrd_status_t lrd_gemm_tuning(int blocks_per_mma);
 
+/* lrd_tucker2_bwd enqueues its independent launches side by side (the dB + dbias product from the start, the
+ * core's filter gradient once dZ2 exists, both on streams the library owns; the data path and dA on the
+ * caller's stream, which waits for the others before the call returns) when `on` is non-zero - the default -
+ * and one after the other on the caller's stream when it is zero.  Same results either way.  With the default,
+ * make the first backward call on a device outside any stream capture (it creates the streams).  Process-wide;
+ * no counterpart in the paper. */
+lrd_status_t lrd_tucker2_overlap(int on);
+
 /* Synchronises the current device, then reports and clears the device-side timeout flag:
  * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
 lrd_status_t lrd_check_device_status(void);

@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_gemm_tuning", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd",
 ]
 
 
@@ -68,6 +68,8 @@ _lib.lrd_linear_group_bwd.restype = _int
 _lib.lrd_linear_group_bwd.argtypes = [_int, C.POINTER(lrd_linear_desc_t)] + [_pp] * 9 + [_int, _pp, C.POINTER(C.c_size_t), C.c_void_p]
 _lib.lrd_gemm_tuning.restype = _int
 _lib.lrd_gemm_tuning.argtypes = [_int]
+_lib.lrd_tucker2_overlap.restype = _int
+_lib.lrd_tucker2_overlap.argtypes = [_int]
 _lib.lrd_check_device_status.restype = _int
 _lib.lrd_check_device_status.argtypes = []
 _lib.lrd_linear_workspace_bytes.restype = _sz
@@ -173,6 +175,10 @@ def lrd_chain_tuning(cluster_blocks=0, kblocks_per_stage=0, chunk_columns=0):
 
 def lrd_gemm_tuning(blocks_per_mma=0):
     _check(_lib.lrd_gemm_tuning(blocks_per_mma))
+
+
+def lrd_tucker2_overlap(on=True):
+    _check(_lib.lrd_tucker2_overlap(int(bool(on))))
 
 
 def lrd_check_device_status():

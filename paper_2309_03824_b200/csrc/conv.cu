@@ -2,6 +2,7 @@
 // backward pass through them under a freeze mask.
 #include "conv.cuh"
 
+#include "streams.cuh"
 #include "tc.cuh"
 
 namespace lrd {
@@ -22,18 +23,29 @@ Tk parse(const lrd_tucker2_desc_t* d) {
 
 size_t act_bytes(const Tk& t, int64_t ch) { return align_up((size_t)(t.P > 0 ? t.P : 1) * ch * elem_size(t.dt), 256); }
 
-size_t split_bytes(const Tk& t) {
-    if (t.P < 1) return 0;
-    size_t need = colsum_scratch_bytes(t.P, t.S);
+// Scratch of the three weight-gradient launches of the backward pass, one region each: they may run side by side.
+struct Scratch { size_t dB, dA, filter; };
+
+Scratch split_regions(const Tk& t) {
+    Scratch r{0, 0, 0};
+    if (t.P < 1) return r;
+    r.dB = colsum_scratch_bytes(t.P, t.S);
     if (t.dt == LRD_BF16) {
-        const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P), b = tc_split_workspace_bytes(t.C, t.r1, t.P);
-        need = need > a ? need : a;
-        need = need > b ? need : b;
-        const size_t f = tc_conv_filter_scratch_bytes(t.B, t.H, t.W, t.r1, t.r2);
-        need = need > f ? need : f;
+        const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P);
+        r.dB = r.dB > a ? r.dB : a;
+        r.dA = tc_split_workspace_bytes(t.C, t.r1, t.P);
+        r.filter = tc_conv_filter_scratch_bytes(t.B, t.H, t.W, t.r1, t.r2);
     }
-    return need;
+    r.dB = align_up(r.dB, 256); r.dA = align_up(r.dA, 256); r.filter = align_up(r.filter, 256);
+    return r;
 }
+
+size_t split_bytes(const Tk& t) {
+    const Scratch r = split_regions(t);
+    return r.dB + r.dA + r.filter;
+}
+
+bool g_tucker_overlap = true;
 
 #define LRD_TRY(expr)                          \
     do {                                       \
@@ -96,30 +108,60 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
 
     void* dZ1 = ws;
     void* dZ2 = (uint8_t*)ws + act_bytes(t, t.r1);
-    float* partials = (float*)((uint8_t*)ws + act_bytes(t, t.r1) + act_bytes(t, t.r2));
-    const size_t pbytes = ws_bytes - act_bytes(t, t.r1) - act_bytes(t, t.r2);
+    const Scratch reg = split_regions(t);
+    uint8_t* scratch0 = (uint8_t*)ws + act_bytes(t, t.r1) + act_bytes(t, t.r2);
+    float* pB = (float*)scratch0;
+    float* pA = (float*)(scratch0 + reg.dB);
+    float* pF = (float*)(scratch0 + reg.dB + reg.dA);
+    (void)ws_bytes;
 
-    LRD_TRY(run_gemm(make_gemm(t.P, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
-    // transposed core + first 1x1 (dX = dZ1 A^T) in one launch where the shape allows; dZ1 is written only for dA
-    const bool fuse_dx = dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
-                         tc_conv_chain_eligible(true, t.B, t.H, t.W, t.r1, t.r2, t.C, t.dt, dZ2, G, A, dX, factors ? dZ1 : nullptr);
-    if (fuse_dx) LRD_TRY(tc_conv3x3_chain(true, dZ2, G, A, nullptr, dX, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.r1, t.r2, t.C, s));
-    else if (dX || factors) LRD_TRY(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
-    if (dX && !fuse_dx) LRD_TRY(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
-    if (factors) {
+    // What depends on what: dZ2 = dY Bm first; the transposed core (+ dX) and the filter gradient both need dZ2 and
+    // nothing of each other; dB (+ db) needs only dY and Z2_save; dA needs the dZ1 the transposed core writes.  Every
+    // launch here is a few microseconds of latency around little work, so the independent ones run side by side:
+    // dB from the start and the filter gradient after dZ2 on library-owned streams, the data path and dA on the
+    // caller's stream, which waits for the other two before this function returns.
+    SideStreams* ss = g_tucker_overlap && (factors || core) ? side_streams() : nullptr;
+    cudaStream_t sB = ss && factors ? ss->aux[0] : s, sF = ss && core ? ss->aux[1] : s;
+    lrd_status_t st = LRD_OK;
+    auto keep = [&st](lrd_status_t x) { if (st == LRD_OK) st = x; };
+    if (sB != s) {
+        if (!stream_after(sB, s, ss->fork)) return LRD_ERR_CUDA;
+    }
+    auto launch_dB = [&]() {
         GemmArgs gb = make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt);
         bool db_done = false;
         if (dbias && path != LRD_PATH_GENERAL) {          // the bias gradient rides on the dB product (A = dY)
             gb.a_colsum = dbias;
             if (tc_gemm_colsum_ok(gb)) db_done = true; else gb.a_colsum = nullptr;
         }
-        LRD_TRY(run_gemm(gb, path, true, partials, pbytes, s));
-        LRD_TRY(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, partials, pbytes, s));
-        if (dbias && !db_done) LRD_TRY(colsum(dY, t.S, t.P, t.S, dbias, t.dt, partials, pbytes, s));
+        keep(run_gemm(gb, path, true, pB, reg.dB, sB));
+        if (dbias && !db_done) keep(colsum(dY, t.S, t.P, t.S, dbias, t.dt, pB, reg.dB, sB));
+    };
+    if (factors && sB != s) launch_dB();
+
+    keep(run_gemm(make_gemm(t.P, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
+    if (core && sF != s) {
+        if (!stream_after(sF, s, ss->mid)) keep(LRD_ERR_CUDA);
+        else keep(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, pF, reg.filter, sF));
     }
-    if (core) LRD_TRY(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, partials, pbytes, s));
-    return LRD_OK;
+    // transposed core + first 1x1 (dX = dZ1 A^T) in one launch where the shape allows; dZ1 is written only for dA
+    const bool fuse_dx = dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+                         tc_conv_chain_eligible(true, t.B, t.H, t.W, t.r1, t.r2, t.C, t.dt, dZ2, G, A, dX, factors ? dZ1 : nullptr);
+    if (fuse_dx) keep(tc_conv3x3_chain(true, dZ2, G, A, nullptr, dX, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.r1, t.r2, t.C, s));
+    else if (dX || factors) keep(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    if (dX && !fuse_dx) keep(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
+    if (factors) {
+        if (sB == s) launch_dB();
+        keep(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, pA, reg.dA, s));
+    }
+    if (core && sF == s) keep(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, pF, reg.filter, s));
+    // join even after a failed launch, so that a capture in progress is left whole
+    if (sB != s && !stream_after(s, sB, ss->aux_done[0])) keep(LRD_ERR_CUDA);
+    if (sF != s && !stream_after(s, sF, ss->aux_done[1])) keep(LRD_ERR_CUDA);
+    return st;
 }
+
+void tucker2_overlap(bool on) { g_tucker_overlap = on; }
 
 // Core convolution dispatch: tensor-core implicit GEMM where the geometry qualifies, else the general kernels.
 lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,

@@ -14,6 +14,10 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
                          void* dB, void* dbias, lrd_tucker_freeze_t freeze, void* ws, size_t ws_bytes, int path,
                          cudaStream_t s);
 
+// Whether the independent launches of tucker2_bwd run side by side on library-owned streams (default) or one
+// after the other on the caller's stream.
+void tucker2_overlap(bool on);
+
 // General-path 3x3 core (stride 1, zero pad 1), NHWC, any channel counts.
 //   fwd:        out[p][o] = sum_{kh,kw,i} in[p + (kh-1, kw-1)][i] G[o][kh][kw][i]
 //   bwd_data:   din[p][i] = sum_{kh,kw,o} dout[p - (kh-1, kw-1)][o] G[o][kh][kw][i]

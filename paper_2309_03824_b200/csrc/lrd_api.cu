@@ -7,6 +7,7 @@
 #include "chain.cuh"
 #include "common.cuh"
 #include "conv.cuh"
+#include "streams.cuh"
 #include "tc.cuh"
 
 using namespace lrd;
@@ -214,6 +215,11 @@ lrd_status_t lrd_gemm_tuning(int blocks_per_mma) {
     return LRD_OK;
 }
 
+lrd_status_t lrd_tucker2_overlap(int on) {
+    tucker2_overlap(on != 0);
+    return LRD_OK;
+}
+
 lrd_status_t lrd_check_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return LRD_ERR_CUDA;
     bool raised = false;
@@ -363,42 +369,8 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
 }
 
 // ---- groups of independent layers -------------------------------------------------------------------
-// Side streams and events of the calling device, made on first use and kept.  Layer 0 of a group runs on the
-// caller's stream, layer i on side stream i - 1; the dU products of a backward group use a second set.
-namespace {
-struct SideStreams {
-    int device = -1;
-    cudaStream_t layer[LRD_MAX_GROUP], du[LRD_MAX_GROUP];
-    cudaEvent_t fork, join[LRD_MAX_GROUP], du_done[LRD_MAX_GROUP];
-};
-SideStreams g_sides[16];
-int g_n_sides = 0;
-
-SideStreams* side_streams() {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
-    for (int i = 0; i < g_n_sides; ++i)
-        if (g_sides[i].device == dev) return &g_sides[i];
-    if (g_n_sides == 16) return nullptr;
-    SideStreams* ss = &g_sides[g_n_sides];
-    bool ok = cudaEventCreateWithFlags(&ss->fork, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; i < LRD_MAX_GROUP && ok; ++i) {
-        ok = cudaStreamCreateWithFlags(&ss->layer[i], cudaStreamNonBlocking) == cudaSuccess &&
-             cudaStreamCreateWithFlags(&ss->du[i], cudaStreamNonBlocking) == cudaSuccess &&
-             cudaEventCreateWithFlags(&ss->join[i], cudaEventDisableTiming) == cudaSuccess &&
-             cudaEventCreateWithFlags(&ss->du_done[i], cudaEventDisableTiming) == cudaSuccess;
-    }
-    if (!ok) return nullptr;
-    ss->device = dev;
-    ++g_n_sides;
-    return ss;
-}
-
-inline bool after(cudaStream_t waiter, cudaStream_t done, cudaEvent_t ev) {      // waiter's next work follows done's work so far
-    return cudaEventRecord(ev, done) == cudaSuccess && cudaStreamWaitEvent(waiter, ev, 0) == cudaSuccess;
-}
-}  // namespace
-
+// Layer 0 of a group runs on the caller's stream, layer i on side stream i - 1; the dU products of a backward
+// group use the auxiliary set.
 lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
                                   const void* const* U, const void* const* bias, void* const* Y, void* const* Z_save,
                                   lrd_freeze_t freeze, void* const* workspace, const size_t* workspace_bytes,
@@ -421,7 +393,7 @@ lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const v
         const lrd_status_t sti = linear_fwd_on(&descs[i], X[i], V[i], U[i], bias ? bias[i] : nullptr, Y[i],
                                                Z_save ? Z_save[i] : nullptr, freeze, workspace[i], workspace_bytes[i], si, share);
         if (sti != LRD_OK) st = sti;
-        if (i > 0 && !after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;      // joined even after a failure
+        if (i > 0 && !stream_after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;      // joined even after a failure
     }
     return st;
 }
@@ -450,15 +422,15 @@ lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const v
     lrd_status_t st = LRD_OK;
     for (int i = 0; i < n; ++i) {
         cudaStream_t si = i == 0 ? s : ss->layer[i - 1];
-        cudaStream_t sd = du_aside ? ss->du[i] : nullptr;
+        cudaStream_t sd = du_aside ? ss->aux[i] : nullptr;
         if (i > 0 && cudaStreamWaitEvent(si, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
         if (sd && cudaStreamWaitEvent(sd, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
         const lrd_status_t sti = linear_bwd_on(&descs[i], dY[i], at(X, i), V[i], U[i], at(Z_save, i), at_w(dX, i), at_w(dU, i),
                                                at_w(dV, i), at_w(dbias, i), freeze, workspace[i], workspace_bytes[i], si, sd,
-                                               ss->du_done[i], share);
+                                               ss->aux_done[i], share);
         if (sti != LRD_OK) st = sti;
-        if (sd && !after(s, sd, ss->du_done[i])) st = LRD_ERR_CUDA;
-        if (i > 0 && !after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;
+        if (sd && !stream_after(s, sd, ss->aux_done[i])) st = LRD_ERR_CUDA;
+        if (i > 0 && !stream_after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;
     }
     return st;
 }

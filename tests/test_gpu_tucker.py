@@ -73,6 +73,26 @@ def test_tensor_core_path(geom, freeze):
     check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 500 + C), freeze)
 
 
+@pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 5, 7, 12, 10, 5, 6)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_backward_launches_side_by_side_or_in_a_row_give_the_same_bits(geom, freeze):
+    """The weight-gradient launches run beside the data path by default; in a row they must give the same results,
+    and a backward repeated back to back (each call joins its side streams before it returns) must not change them."""
+    B, H, W, C, S, r1, r2 = geom
+    case = wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 600 + C)
+    try:
+        b.lrd_tucker2_overlap(False)
+        row = run_tucker(case, freeze)
+    finally:
+        b.lrd_tucker2_overlap(True)
+    check_tucker(case, freeze)
+    for _ in range(3):
+        side = run_tucker(case, freeze)
+        for k, v in side.items():
+            if v is not None:
+                assert torch.equal(v, row[k]), k
+
+
 @pytest.mark.parametrize("freeze", [b.LRD_TK_FREEZE_CORE, b.LRD_TK_FREEZE_FACTORS])
 def test_c3_resnet_stage3_shape_full_size(freeze):
     c = wl.C3_TUCKER

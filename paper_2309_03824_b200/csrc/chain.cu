@@ -36,6 +36,8 @@ using namespace ptx;
 
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 12;
+constexpr int kMaxCluster = 4;       // blocks per row tile
+constexpr int kMaxKb2 = 8;           // 64-column k-blocks of T (r <= 512)
 constexpr uint32_t kSmemLimit = 224 * 1024;         // dynamic shared memory; the rest is left for the barriers and the bias
 constexpr uint32_t kInTileBytes = 128 * 64 * 2;     // In tile of one k-block: 128 rows x 64 k
 constexpr uint32_t kSlabBytes = 32 * 32 * 2;        // epilogue slab of one warp: 32 rows x 32 columns of bf16
@@ -50,6 +52,9 @@ struct ChainParams {
     const __nv_bfloat16* bias;
     int has_tsave;
     unsigned int* timeout_flag;
+    // Phase 2 of block c walks over the 64-column k-blocks of T in the order kb_order[c] (4 bits per position)
+    // and needs the slices in kb_slices[c] (a 4-bit mask per position) for the k-block at that position.
+    uint32_t kb_order[kMaxCluster], kb_slices[kMaxCluster];
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -58,7 +63,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
              const __grid_constant__ CUtensorMap tmT, const ChainParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages],
-        tacc_bar, tready_bar, out_full[2], out_empty[2];
+        tacc_bar, tready_bar[kMaxCluster], out_full[2], out_empty[2];
     __shared__ __align__(16) float bias_s[2][256];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -77,6 +82,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0);
     const int lane = threadIdx.x % 32;
     const int c = (int)cluster_ctarank();
+    const uint32_t my_order = c == 0 ? p.kb_order[0] : (c == 1 ? p.kb_order[1] : (c == 2 ? p.kb_order[2] : p.kb_order[3]));
+    const uint32_t my_slices = c == 0 ? p.kb_slices[0] : (c == 1 ? p.kb_slices[1] : (c == 2 ? p.kb_slices[2] : p.kb_slices[3]));
     const int m0 = blockIdx.y * 128;
     const int ng1 = (p.kb1 + p.G1 - 1) / p.G1;                                 // stage turns of phase 1
     // phase-1 stage: G1 In tiles, then the P boxes (one per column atom, 64 G1 rows tall)
@@ -98,13 +105,15 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         prefetch_tmap(&tmQ);
         prefetch_tmap(&tmOut);
         mbar_init(smem_u32(&tacc_bar), 1);
-        // T complete = this block's own slice written (one arrival) + the peers' slices landed (bytes)
-        mbar_init(smem_u32(&tready_bar), 2);
+        // one barrier per slice of T: this block's own slice is ready after one arrival (written by its gather
+        // warps), a peer's slice once its bytes have landed
+        for (int j = 0; j < p.C; ++j) mbar_init(smem_u32(&tready_bar[j]), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&out_full[i]), 1);
             mbar_init(smem_u32(&out_empty[i]), 4);
         }
-        mbar_expect_tx(smem_u32(&tready_bar), (uint32_t)(p.C - 1) * 256u * (uint32_t)p.RS);
+        for (int j = 0; j < p.C; ++j)
+            if (j != c) mbar_expect_tx(smem_u32(&tready_bar[j]), 256u * (uint32_t)p.RS);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -155,7 +164,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         s = 0;
         ph = 1;
         for (int j = c; j < p.n_chunks && ok; j += p.C) {
-            for (int kb = 0; kb < p.kb2; ++kb) {             // columns past r read as zeros (never multiplied)
+            for (int i = 0; i < p.kb2; ++i) {                // columns past r read as zeros (never multiplied)
+                const int kb = (int)((my_order >> (4 * i)) & 15u);
                 const uint32_t fb = smem_u32(&full2[s]);
                 ok = mbar_wait_uniform(smem_u32(&empty2[s]), ph, ab);
                 if (!ok) break;
@@ -205,9 +215,11 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         if (ok && elect_one()) mma_commit(smem_u32(&tacc_bar));
         __syncwarp();
         if (lane == 0) { LRD_TS(7); }
-        // every slice of T has landed in this block's buffer (which also means the phase-1 accumulator
-        // columns have been read out)
-        if (ok) ok = mbar_wait_cluster_uniform(smem_u32(&tready_bar), 0, ab);
+        // this block's own slice is in its T buffer, which also means that the phase-1 accumulator columns
+        // (which the first chunk's accumulator overlaps) have been read out; the peers' slices are waited for
+        // where the k-loop first touches them
+        if (ok) ok = mbar_wait_uniform(smem_u32(&tready_bar[c]), 0, ab);
+        uint32_t slices_ready = 1u << c;
         if (lane == 0) { LRD_TS(8); }
         const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
         const uint64_t t_desc0 = smem_desc(t_base, 0, 8u * t_sw, t_sw);
@@ -217,31 +229,45 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         for (int j = c; j < p.n_chunks && ok; j += p.C, ++i2) {
             const uint32_t d_tmem = tmem_base + (uint32_t)(i2 & 1) * 256u;
             ok = mbar_wait_uniform(smem_u32(&out_empty[i2 & 1]), ((i2 >> 1) & 1) ^ 1, ab);   // accumulator buffer drained
-            for (int kb = 0; kb < p.kb2 && ok; ++kb) {
+            for (int i = 0; i < p.kb2 && ok; ++i) {
+                const int kb = (int)((my_order >> (4 * i)) & 15u);
+                const int nks = min(4, p.ks2 - kb * 4);
+                if (i2 == 0) {
+                    uint32_t need = ((my_slices >> (4 * i)) & 15u) & ~slices_ready;
+                    while (need && ok) {
+                        const int j = __ffs(need) - 1;
+                        ok = mbar_wait_cluster_uniform(smem_u32(&tready_bar[j]), 0, ab);
+                        need &= need - 1;
+                        slices_ready |= 1u << j;
+                    }
+                    if (!ok) break;
+                }
                 ok = mbar_wait_uniform(smem_u32(&full2[s]), ph, ab);
                 if (!ok) break;
-                if (i2 == 0 && kb < 8 && lane == 0) { LRD_TS(24 + kb); }
+                if (i2 == 0 && i < 8 && lane == 0) { LRD_TS(24 + i); }
                 tc_fence_after();
                 const uint32_t q_src = ring2_base + s * p.stage2_bytes;
                 const uint64_t bd = a_desc0 + ((q_src >> 4) & 0x3FFFu);
-                const int nks = min(4, p.ks2 - kb * 4);
                 if (elect_one()) {
                     for (int kk = 0; kk < nks; ++kk) {
                         const uint32_t ks = (uint32_t)(kb * 4 + kk);      // 16-column step within T
                         const uint64_t ad = t_desc0 + (((ks >> p.t_steps_lg) * t_atom_bytes + (ks & ((1u << p.t_steps_lg) - 1u)) * 32u) >> 4);
-                        mma_bf16_ss(d_tmem, ad, bd + 2u * kk, idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
+                        mma_bf16_ss(d_tmem, ad, bd + 2u * kk, idesc2, (i > 0 || kk > 0) ? 1u : 0u);
                     }
                     mma_commit(smem_u32(&empty2[s]));
-                    if (kb == p.kb2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
+                    if (i == p.kb2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
                 }
                 __syncwarp();
-                if (i2 == 0 && kb < 8 && lane == 0) { LRD_TS(32 + kb); }
+                if (i2 == 0 && i < 8 && lane == 0) { LRD_TS(32 + i); }
                 if (++s == p.S2) { s = 0; ph ^= 1; }
             }
         }
         if (lane == 0) { LRD_TS(9); }
+        // a block without a chunk of its own still has to have received every slice before it passes barrier 2
+        for (int j = 0; j < p.C && ok; ++j)
+            if (!((slices_ready >> j) & 1u)) ok = mbar_wait_cluster_uniform(smem_u32(&tready_bar[j]), 0, ab);
         cluster_wait();        // barrier 1 (long complete: every peer has pushed into this block)
-        cluster_arrive_relaxed();   // barrier 2: this block has received everything its peers send (T was complete above)
+        cluster_arrive_relaxed();   // barrier 2: this block has received everything its peers send
     } else {
         // ------------------------------------------------------------------ gather + epilogue
         const int q = warp % 4;                              // tensor-memory lanes [32 q, 32 q + 32)
@@ -291,9 +317,9 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;
                 for (int t = 1; t < p.C; ++t) {
                     const uint32_t peer = (uint32_t)((c + t) % p.C);
-                    dsmem_bulk_copy(slice, slice, 256u * (uint32_t)p.RS, smem_u32(&tready_bar), peer);
+                    dsmem_bulk_copy(slice, slice, 256u * (uint32_t)p.RS, smem_u32(&tready_bar[c]), peer);
                 }
-                mbar_arrive(smem_u32(&tready_bar));
+                mbar_arrive(smem_u32(&tready_bar[c]));
                 if (p.has_tsave) {
                     for (int a = 0; a * p.taw < p.RS; ++a)
                         tma_store_2d(&tmT, slice + (uint32_t)a * t_atom_bytes, c * p.RS + a * p.taw, m0);
@@ -547,6 +573,29 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     p.t_steps_lg = p.taw == 64 ? 2 : (p.taw == 32 ? 1 : 0);
     p.bias = (const __nv_bfloat16*)a.bias;
     p.has_tsave = a.T_save ? 1 : 0;
+    // A block sends its slice of T to the peers c + 1, c + 2, ... in turn, so slice j reaches block c as the
+    // ((c - j) mod C)-th arrival (0 = its own); phase 2 takes the k-blocks in the order in which the last slice
+    // they touch arrives.  The order depends on the launch shape only, so results stay reproducible.
+    for (int c = 0; c < kMaxCluster; ++c) {
+        p.kb_order[c] = 0; p.kb_slices[c] = 0;
+        if (c >= p.C) continue;
+        int n = 0;
+        for (int rank = 0; rank < p.C; ++rank)
+            for (int kb = 0; kb < p.kb2; ++kb) {
+                const int nks = std::min(4, p.ks2 - kb * 4);
+                const int j_lo = kb * 64 / p.RS, j_hi = (kb * 64 + nks * 16 - 1) / p.RS;
+                int worst = 0;
+                uint32_t mask = 0;
+                for (int j = j_lo; j <= j_hi; ++j) {
+                    worst = std::max(worst, (c - j + p.C) % p.C);
+                    mask |= 1u << j;
+                }
+                if (worst != rank) continue;
+                p.kb_order[c] |= (uint32_t)kb << (4 * n);
+                p.kb_slices[c] |= mask << (4 * n);
+                ++n;
+            }
+    }
     p.timeout_flag = device_timeout_flag();
 
     static bool configured = false;

@@ -1,6 +1,6 @@
 """Groups of independent layers enqueued side by side (the query / key / value projections of an attention block):
-parity of every layer with the oracle, identity with the single-layer calls, replay from a CUDA graph, and the
-argument checks that run before anything is enqueued."""
+parity of every layer with the oracle, agreement with the single-layer calls, replay from a CUDA graph (same bits
+every time), and the argument checks that run before anything is enqueued."""
 import numpy as np
 import pytest
 import torch
@@ -58,9 +58,14 @@ class Group:
                     continue
                 got = self.out[name][li]
                 assert rel_err(got, ref[name]) <= TOL["bf16"], (li, name)
-                # a group changes where and beside what a layer runs, not what is summed in which order
+                # A group changes where and beside what a layer runs.  The intermediate and the weight gradients are
+                # summed in the same order as in a single-layer call (same bits); the second product of a chain walks
+                # over the rank in an order that depends on the cluster size, so Y and dX agree to rounding only.
                 if one is not None and one[name] is not None:
-                    assert torch.equal(got, one[name]), (li, name)
+                    if name in ("Y", "dX"):
+                        assert rel_err(got, host(one[name])) <= 2.0 ** -7, (li, name)
+                    else:
+                        assert torch.equal(got, one[name]), (li, name)
 
 
 QKV = [(520, 264, 264, 64)] * 3

@@ -30,7 +30,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture of
 # the 768->3072, r=384 forward; summary in profiles/chain_kernel_ffn1_forward.md).  It is reported only while the
 # kernel's sources still have the digest the capture was taken with.
-NCU_TRAFFIC = {"digest": "5cf3793f6d951448", "bytes_per_launch": 9315328}
+NCU_TRAFFIC = {"digest": "4ada81cd16d2e7b7", "bytes_per_launch": 9319168}
 KERNEL_SOURCES = ("paper_2309_03824_b200/csrc/chain.cu", "paper_2309_03824_b200/csrc/ptx.cuh")
 
 

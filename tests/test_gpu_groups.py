@@ -136,3 +136,22 @@ def test_group_checks_every_layer_before_enqueueing_anything():
     g.fwd()
     g.bwd()
     g.check(single=False)
+
+
+def _svd_factors(W, r):
+    Uf, s, Vt = np.linalg.svd(W, full_matrices=False)     # input construction only
+    root = np.sqrt(s[:r])
+    return Vt[:r].T * root, Uf[:, :r] * root
+
+
+@pytest.mark.parametrize("freeze", [b.LRD_FREEZE_U, b.LRD_FREEZE_V])
+def test_bert_base_attention_projections_as_the_benchmark_launches_them(freeze):
+    """attn_q / attn_k / attn_v at full size (4096 tokens, 768 -> 768, r = 192, factors from an SVD) as one group:
+    the launch configuration of the benchmark step, every output element against the oracle."""
+    cases = []
+    for idx, (name, K, N, r) in enumerate(wl.C1_BERT_LAYERS[:3]):
+        cases.append(wl.linear_case(wl.C1_M, K, N, r, "bf16", 1000 + 10 * idx, wl.W_STD_TRANSFORMER, _svd_factors))
+    g = Group(cases, freeze)
+    g.fwd()
+    g.bwd()
+    g.check(single=False)

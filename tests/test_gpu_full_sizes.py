@@ -52,3 +52,10 @@ def test_rank_sweep_layer_full_size(r, freeze):
 def test_gpt2_medium_shaped_layers_full_size(layer, freeze):
     name, K, N, r = layer
     check_sampled(wl.random_factor_case(wl.C4_M, K, N, r, "bf16", 4000 + K + r), freeze)
+
+
+@pytest.mark.parametrize("r", [64, 72])
+def test_quarter_of_a_million_tokens(r):
+    """2049 row tiles with a ragged last one, weight gradients summed over 262 221 tokens (4098 k-blocks of 64):
+    r = 64 takes the fused chain, r = 72 (not a multiple of 16) the separate products on pairs of SMs."""
+    check_sampled(wl.random_factor_case(262221, 136, 264, r, "bf16", 5000 + r), b.LRD_FREEZE_NONE)

@@ -144,8 +144,8 @@ lrd_status_t lrd_gemm_tuning(int blocks_per_mma);
  * core's filter gradient once dZ2 exists, both on streams the library owns; the data path and dA on the
  * caller's stream, which waits for the others before the call returns) when `on` is non-zero - the default -
  * and one after the other on the caller's stream when it is zero.  Same results either way.  With the default,
- * make the first backward call on a device outside any stream capture (it creates the streams).  Process-wide;
- * no counterpart in the paper. */
+ * make a host thread's first backward call on a device outside any stream capture (it creates that thread's
+ * streams).  The switch is process-wide; no counterpart in the paper. */
 lrd_status_t lrd_tucker2_overlap(int on);
 
 /* Synchronises the current device, then reports and clears the device-side timeout flag:
@@ -195,17 +195,18 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
  * them up where the layers share X).  One mask applies to the whole group.
  *
  * The layers are enqueued side by side: layer 0 on `cuda_stream`, the others on streams the library
- * owns (created on first use, one set per device, never freed), which start after the work already in
+ * owns (created on first use, one set per host thread and device, never freed), which start after the work already in
  * `cuda_stream` and which `cuda_stream` waits for before the call returns - so to the caller the group
  * behaves like n single-layer calls on `cuda_stream`, and it may be captured into a CUDA graph.  Each
  * launch is shaped for 1/n of the SMs.  In the backward, a layer's dU (+ dbias) product runs beside its
- * data chain.  Results are those of the single-layer calls.  n = 1 is allowed (then only the dU
- * overlap differs from lrd_linear_bwd).
+ * data chain.  Z_save, dU, dV and dbias have the bits of the single-layer calls; Y and dX agree with them to
+ * rounding (the fused kernel sums over the rank in an order that depends on its cluster size, which follows
+ * the launch's share of the SMs).  n = 1 is allowed (then only the dU overlap differs from lrd_linear_bwd).
  *
  * Errors: LRD_ERR_INVALID_ARG for n outside [0, LRD_MAX_GROUP] or a NULL required array; otherwise the
- * first failing layer's status.  All layers are validated before anything is enqueued.  Not
- * thread-safe: two host threads must not run groups on the same device at the same time.  Make the
- * first group call on a device outside any stream capture (it creates the library's streams). */
+ * first failing layer's status.  All layers are validated before anything is enqueued.  Every host
+ * thread has its own set of library streams, so groups may run from several threads at once.  Make a
+ * thread's first group call on a device outside any stream capture (it creates that set). */
 #define LRD_MAX_GROUP 8
 lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
                                   const void* const* U, const void* const* bias, void* const* Y, void* const* Z_save,

@@ -3,8 +3,9 @@
 namespace lrd {
 namespace {
 constexpr int kMaxDevices = 16;
-SideStreams g_sides[kMaxDevices];
-int g_n_sides = 0;
+// one table per host thread: calls from different threads never share a stream or an event
+thread_local SideStreams g_sides[kMaxDevices];
+thread_local int g_n_sides = 0;
 }  // namespace
 
 SideStreams* side_streams() {

@@ -1,8 +1,8 @@
-// Streams and events the library owns, for work that runs beside the caller's stream: one set per device,
-// made on first use (outside any stream capture) and kept until the process exits.  Side work starts after
+// Streams and events the library owns, for work that runs beside the caller's stream: one set per host thread
+// and device, made on that thread's first use (outside any stream capture) and kept until the process exits.  Side work starts after
 // the caller's earlier work (fork) and the caller's stream waits for it before the entry point returns (join),
 // so to the caller every entry point stays ordered on its own stream, and the pattern can be captured
-// into a CUDA graph.  Not thread-safe: the events are shared by all calls on a device.
+// into a CUDA graph.  Host threads do not share sets, so calls from different threads do not interfere.
 #pragma once
 #include "common.cuh"
 

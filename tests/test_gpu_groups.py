@@ -155,3 +155,31 @@ def test_bert_base_attention_projections_as_the_benchmark_launches_them(freeze):
     g.fwd()
     g.bwd()
     g.check(single=False)
+
+
+def test_groups_from_two_host_threads_at_once():
+    """Every host thread has its own library streams: two threads, each with its own stream, run groups at the same
+    time (the C calls release the interpreter lock), many times over; each must get its own right answers."""
+    import threading
+    gs = [Group(make_group(QKV, 1700 + 50 * t, shared_x=True), b.LRD_FREEZE_NONE) for t in range(2)]
+    errors = []
+
+    def work(g):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                for _ in range(20):
+                    g.fwd()
+                    g.bwd()
+            st.synchronize()
+        except Exception as e:          # surfaced in the main thread below
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(g,)) for g in gs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for g in gs:
+        g.check(single=False)

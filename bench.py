@@ -239,6 +239,7 @@ def main():
                     help="qkv: the three independent attention projections go out as one group (the default); none: one call per layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every step instead of CUDA graphs")
+    ap.add_argument("--single-step-graphs", action="store_true", help="one CUDA graph per step instead of one per cycle of steps (every buffer set under both masks)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -357,6 +358,21 @@ def main():
                 graphs[(s, f)] = g
         torch.cuda.synchronize()
 
+    # One graph for a whole cycle of steps (every buffer set once, under both masks = 2 S steps): the dependent-launch
+    # overlap then also holds across step boundaries, and the cost of a graph launch (about 10 us of device idle time
+    # between two replays) is paid once per cycle.  Steps that do not fill a cycle replay the single-step graphs.
+    cycle = 2 * S
+    cycle_graph = None
+    if graphs and not args.single_step_graphs:
+        side = torch.cuda.Stream()
+        cycle_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(cycle_graph, stream=side):
+                for s in range(S):
+                    step_eager(s, masks[0])
+                    step_eager(s, masks[1])
+        torch.cuda.synchronize()
+
     def step(i):
         s, f = (i // 2) % S, masks[i % 2]
         if graphs:
@@ -364,18 +380,32 @@ def main():
         else:
             step_eager(s, f)
 
+    def run_steps(start, n):
+        """Steps start .. start + n - 1, exactly n of them."""
+        i, end = start, start + n
+        while i < end:
+            if cycle_graph is not None and i % cycle == 0 and i + cycle <= end:
+                cycle_graph.replay()
+                i += cycle
+            else:
+                step(i)
+                i += 1
+
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
+    def timed(fn, steps, bulk=False):
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.time()
         e0.record()
-        for i in range(steps):
-            fn(i)
+        if bulk:
+            fn(0, steps)
+        else:
+            for i in range(steps):
+                fn(i)
         e1.record()
         torch.cuda.synchronize()
         t1 = time.time()
@@ -389,17 +419,15 @@ def main():
         t_wait = time.time()
         while not sampler.rows and time.time() - t_wait < 5.0:      # nvidia-smi takes a moment to print its first sample
             time.sleep(0.05)
-    for i in range(args.warmup):
-        step(i)
-    ms, t0, t1 = timed(step, args.steps)
+    run_steps(0, args.warmup)
+    ms, t0, t1 = timed(run_steps, args.steps, bulk=True)
     # The timed region is shorter than one sampling period (K steps of ~0.2 ms): the same steps go on, untimed, for
     # about a second and a half so that the clock samples are taken under this very load.
     if rank == 0:
         i = args.steps
         while time.time() - t1 < 1.5:
-            for _ in range(100):
-                step(i)
-                i += 1
+            run_steps(i, 12 * cycle)
+            i += 12 * cycle
             torch.cuda.synchronize()
     barrier()
     clocks = sampler.summary(t0, time.time()) if rank == 0 else None
@@ -407,16 +435,33 @@ def main():
     # the same steps on ONE buffer set (its 239 MB partly stay in L2 from step to step): reported beside the headline, labelled
     hot = None
     if S > 1:
-        def hot_step(i):
-            f = masks[i % 2]
-            if graphs:
-                graphs[(0, f)].replay()
-            else:
-                step_eager(0, f)
-        for i in range(4):
-            hot_step(i)
-        hot_steps = max(2, min(args.steps, 100) // 2 * 2)
-        hms, _, _ = timed(hot_step, hot_steps)
+        hot_graph = None
+        if cycle_graph is not None:              # the same cycle of 2 S steps, all on buffer set 0
+            side = torch.cuda.Stream()
+            hot_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(hot_graph, stream=side):
+                    for _ in range(S):
+                        step_eager(0, masks[0])
+                        step_eager(0, masks[1])
+            torch.cuda.synchronize()
+
+        def hot_steps_run(start, n):
+            i, end = start, start + n
+            while i < end:
+                if hot_graph is not None and i % cycle == 0 and i + cycle <= end:
+                    hot_graph.replay()
+                    i += cycle
+                else:
+                    f = masks[i % 2]
+                    if graphs:
+                        graphs[(0, f)].replay()
+                    else:
+                        step_eager(0, f)
+                    i += 1
+        hot_steps_run(0, cycle)
+        hot_steps = max(2, min(args.steps, 200) // 2 * 2)
+        hms, _, _ = timed(hot_steps_run, hot_steps, bulk=True)
         hot = {"ms_per_step": hms / hot_steps, "steps": hot_steps,
                "note": "one activation buffer set re-used every step (partly L2-resident); not the headline"}
     tokens = wl.C1_M * world
@@ -573,7 +618,8 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": config_dict({"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                                        "l2": f"cycling {S} activation buffer sets, {S * act_bytes_per_set / 1e6:.0f} MB > 126 MB L2",
-                                       "launch": "eager C-ABI calls" if args.no_graph else "CUDA graph replay of the C-ABI calls",
+                                       "launch": "eager C-ABI calls" if args.no_graph else ("CUDA graph replay of the C-ABI calls, one graph per step" if args.single_step_graphs
+                                                  else f"CUDA graph replay of the C-ABI calls, one graph per cycle of {cycle} steps (every buffer set under both masks)"),
                                        "path": args.path,
                                        "groups": {"qkv": "attn_q/k/v side by side in one group call, the other layers one call each",
                                                   "none": "one call per layer"}[args.groups]}),

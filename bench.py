@@ -542,7 +542,7 @@ def main():
     roof = None
     kernels = []
     if rank == 0:
-        reps = 40
+        reps, rounds = 10, 8          # 10 replays of a graph of 8 x S launches of the op
 
         def time_op(fn):
             for s in range(S):
@@ -555,8 +555,9 @@ def main():
             g = torch.cuda.CUDAGraph()
             with torch.cuda.stream(side2):
                 with torch.cuda.graph(g, stream=side2):
-                    for s in range(S):
-                        fn(s)
+                    for _ in range(rounds):          # many launches per graph: a graph launch costs ~14 us of idle device
+                        for s in range(S):
+                            fn(s)
             torch.cuda.synchronize()
             g.replay()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -566,7 +567,7 @@ def main():
                 g.replay()
             e1.record()
             torch.cuda.synchronize()
-            return e0.elapsed_time(e1) * 1e-3 / (reps * S), n_k
+            return e0.elapsed_time(e1) * 1e-3 / (reps * rounds * S), n_k
 
         for L in layers[3:]:          # one attention layer and both FFN layers
             M, K, N, r = L["M"], L["K"], L["N"], L["r"]

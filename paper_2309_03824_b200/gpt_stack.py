@@ -126,7 +126,7 @@ def main():
             n0 = b.lrd_launch_count()
             lrd_step(0, f, grouped)
             nk = b.lrd_launch_count() - n0
-            sec = time_graph(lambda s: lrd_step(s, f, grouped), SETS, a.reps)
+            sec = time_graph(lambda s: lrd_step(s, f, grouped), SETS, a.reps, rounds=1)
             rows.append((label + (", q/k/v grouped" if grouped else ", one call per layer"), sec, flops, roof(work), nk))
     work, flops = [], 0
     for name, K, N, r in wl.C4_GPT_LAYERS:
@@ -136,7 +136,7 @@ def main():
     n0 = b.lrd_launch_count()
     dense_step(0)
     nk = b.lrd_launch_count() - n0
-    sec = time_graph(dense_step, SETS, a.reps)
+    sec = time_graph(dense_step, SETS, a.reps, rounds=1)
     rows.append(("undecomposed stack", sec, flops, roof(work), nk))
     if b.lrd_check_device_status() != b.LRD_OK:
         raise SystemExit("device-side wait timed out")

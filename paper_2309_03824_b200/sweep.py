@@ -44,15 +44,16 @@ def dense_work(M, K, N):
     return 6 * M * K * N, 2 * (M * K + K * N + N + M * N) + 2 * (M * N + K * N + M * K) + 2 * (M * K + K * N + N)
 
 
-def time_graph(fn, sets, reps):
+def time_graph(fn, sets, reps, rounds=1):
     for s in range(sets):
         fn(s)
     torch.cuda.synchronize()
     side, g = torch.cuda.Stream(), torch.cuda.CUDAGraph()
     with torch.cuda.stream(side):
         with torch.cuda.graph(g, stream=side):
-            for s in range(sets):
-                fn(s)
+            for _ in range(rounds):          # a graph launch leaves the device idle for ~14 us: more rounds per graph for short steps
+                for s in range(sets):
+                    fn(s)
     torch.cuda.synchronize()
     g.replay()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -62,7 +63,7 @@ def time_graph(fn, sets, reps):
         g.replay()
     e1.record()
     torch.cuda.synchronize()
-    return e0.elapsed_time(e1) * 1e-3 / (reps * sets)
+    return e0.elapsed_time(e1) * 1e-3 / (reps * rounds * sets)
 
 
 def main():

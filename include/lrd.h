@@ -156,8 +156,8 @@ lrd_status_t lrd_check_device_status(void);
  * streams; memset nodes of zero-filled gradients are not counted).  For launch accounting. */
 uint64_t lrd_launch_count(void);
 
-/* Scratch bytes lrd_linear_fwd (is_bwd = 0) or lrd_linear_bwd (is_bwd = 1) needs for this layer and
- * mask, for whichever path the library may take.  0 on a bad descriptor. */
+/* Scratch bytes lrd_linear_fwd (is_bwd = 0), lrd_linear_bwd (is_bwd = 1) or lrd_linear_bwd_accumulate
+ * (is_bwd = 2) needs for this layer and mask, for whichever path the library may take.  0 on a bad descriptor. */
 size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t freeze, int is_bwd);
 size_t lrd_tucker2_workspace_bytes(const lrd_tucker2_desc_t* desc, lrd_tucker_freeze_t freeze, int is_bwd);
 size_t lrd_dense_workspace_bytes(const lrd_linear_desc_t* desc, int is_bwd);
@@ -182,6 +182,16 @@ lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const 
 lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
                             const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                             lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward with gradient accumulation: as lrd_linear_bwd, but the unfrozen factor's dU, dbias and dV are ADDED to
+ * what the buffers hold (gradient accumulation over micro-batches) instead of overwritten; dX is overwritten as
+ * usual.  A frozen factor's gradient buffers are not touched at all (its gradient is zero), and may be NULL.
+ * This step's gradients are formed in scratch at the end of the workspace, rounded to the storage type, then
+ * added in fp32 and rounded once more.  Workspace: lrd_linear_workspace_bytes(desc, freeze, 2).  The paper's
+ * Section 2.2 trains with plain steps; accumulation is a convenience with no counterpart there. */
+lrd_status_t lrd_linear_bwd_accumulate(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                                       const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                                       lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---- groups of independent decomposed layers -------------------------------------------------------
  * The n layers of a group depend on nothing the others produce (the query, key and value projections

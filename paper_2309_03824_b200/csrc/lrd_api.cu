@@ -2,6 +2,7 @@
 // the layer runs in this library's own kernels; nothing here falls back to the host.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 
 #include "chain.cuh"
@@ -72,6 +73,11 @@ GemmArgs gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool 
 
 size_t linear_z_bytes(const Linear& L) { return align_up((size_t)(L.M > 0 ? L.M : 1) * L.r * elem_size(L.dt), 256); }
 
+size_t linear_grad_scratch_bytes(const Linear& L) {     // dU, dV and dbias of one step, in the parameters' layouts
+    const size_t e = elem_size(L.dt);
+    return align_up((size_t)L.N * L.ldu * e, 256) + align_up((size_t)L.K * L.ldv * e, 256) + align_up((size_t)L.N * e, 256);
+}
+
 size_t linear_split_bytes(const Linear& L) {     // scratch after dZ: split partials of dU / dV, partial column sums
     if (L.M < 1) return 0;
     size_t need = colsum_scratch_bytes(L.M, L.N);
@@ -106,6 +112,30 @@ lrd_status_t zero_fill(void* p, int64_t rows, int64_t cols, int64_t ld, lrd_dtyp
     if (!p || rows <= 0 || cols <= 0) return LRD_OK;
     const size_t e = elem_size(dt);
     return cudaMemset2DAsync(p, (size_t)ld * e, 0, (size_t)cols * e, (size_t)rows, s) == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+namespace {
+// dst[row][col] += src[row][col] (both with leading dimension ld): fp32 sum, one rounding to the storage type.
+template <typename T>
+__global__ void add_into_kernel(T* __restrict__ dst, const T* __restrict__ src, int64_t rows, int64_t cols, int64_t ld) {
+    const int64_t n = rows * cols;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t at = (i / cols) * ld + i % cols;
+        dst[at] = (T)((float)dst[at] + (float)src[at]);
+    }
+}
+}  // namespace
+
+lrd_status_t add_into(void* dst, const void* src, int64_t rows, int64_t cols, int64_t ld, lrd_dtype_t dt, cudaStream_t s) {
+    if (!dst || rows <= 0 || cols <= 0) return LRD_OK;
+    const int64_t n = rows * cols;
+    const unsigned blocks = (unsigned)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    if (dt == LRD_BF16)
+        add_into_kernel<<<blocks, 256, 0, s>>>((__nv_bfloat16*)dst, (const __nv_bfloat16*)src, rows, cols, ld);
+    else
+        add_into_kernel<<<blocks, 256, 0, s>>>((float*)dst, (const float*)src, rows, cols, ld);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
 GemmArgs make_gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
@@ -231,7 +261,10 @@ size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t fr
     Linear L;
     if (parse_linear(desc, &L, false) != LRD_OK) return 0;
     (void)freeze;
-    return is_bwd ? linear_z_bytes(L) + linear_split_bytes(L) : linear_z_bytes(L);
+    if (!is_bwd) return linear_z_bytes(L);
+    const size_t bwd = linear_z_bytes(L) + linear_split_bytes(L);
+    if (is_bwd != 2) return bwd;
+    return align_up(bwd, 256) + linear_grad_scratch_bytes(L);      // + one gradient of every kind, for lrd_linear_bwd_accumulate
 }
 
 size_t lrd_dense_workspace_bytes(const lrd_linear_desc_t* desc, int is_bwd) {
@@ -366,6 +399,39 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
                             lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return linear_bwd_on(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, workspace_bytes,
                          (cudaStream_t)cuda_stream, nullptr, nullptr, 0);
+}
+
+lrd_status_t lrd_linear_bwd_accumulate(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                                       const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                                       lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Linear L;
+    LRD_TRY(parse_linear(desc, &L, false));
+    const uint32_t plan = lrd_linear_bwd_plan(freeze);
+    if (!plan) return LRD_ERR_INVALID_ARG;
+    LRD_TRY(check_ws(workspace, workspace_bytes, lrd_linear_workspace_bytes(desc, freeze, 2)));
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // this step's gradients go to scratch behind the ordinary backward workspace, then into the caller's buffers;
+    // a frozen factor's buffers are not touched (its gradient is zero)
+    const size_t bwd_bytes = align_up(lrd_linear_workspace_bytes(desc, freeze, 1), 256);
+    const size_t e = elem_size(L.dt);
+    uint8_t* g = (uint8_t*)workspace + bwd_bytes;
+    void* gU = g;
+    void* gV = g + align_up((size_t)L.N * L.ldu * e, 256);
+    void* gb = g + align_up((size_t)L.N * L.ldu * e, 256) + align_up((size_t)L.K * L.ldv * e, 256);
+    const bool du = (plan & LRD_PLAN_DU) != 0, dv = (plan & LRD_PLAN_DV) != 0;
+    if ((du && !dU) || (dv && !dV)) return LRD_ERR_INVALID_ARG;
+    const void* outs[] = {dU, dV, dbias};
+    for (const void* p : outs)
+        if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
+    LRD_TRY(linear_bwd_on(desc, dY, X, V, U, Z_save, dX, du ? gU : nullptr, dv ? gV : nullptr, (du && dbias) ? gb : nullptr, freeze,
+                          workspace, bwd_bytes, s, nullptr, nullptr, 0));
+    if (L.M == 0) return LRD_OK;
+    if (du) {
+        LRD_TRY(add_into(dU, gU, L.N, L.r, L.ldu, L.dt, s));
+        if (dbias) LRD_TRY(add_into(dbias, gb, 1, L.N, L.N, L.dt, s));
+    }
+    if (dv) LRD_TRY(add_into(dV, gV, L.K, L.r, L.ldv, L.dt, s));
+    return LRD_OK;
 }
 
 // ---- groups of independent layers -------------------------------------------------------------------

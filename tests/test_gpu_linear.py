@@ -7,7 +7,7 @@ from oracle import lrd_oracle as o
 from paper_2309_03824_b200 import binding as b
 from paper_2309_03824_b200 import workloads as wl
 
-from helpers import DT, check_linear, dev, host, rel_err, run_linear, workspace
+from helpers import DT, TOL, check_linear, dev, host, oracle_linear, rel_err, run_linear, workspace
 
 pytestmark = pytest.mark.gpu
 MASKS = [b.LRD_FREEZE_NONE, b.LRD_FREEZE_U, b.LRD_FREEZE_V]
@@ -203,3 +203,42 @@ def test_fused_forward_is_one_kernel_and_keeps_z_on_chip():
         b.lrd_set_path(b.LRD_PATH_AUTO)
     torch.cuda.synchronize()
     assert b.lrd_check_device_status() == b.LRD_OK
+
+
+@pytest.mark.parametrize("dtype,shape", [("bf16", (520, 264, 328, 64)), ("bf16", (300, 200, 136, 72)), ("f32", (256, 96, 80, 24))])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_backward_accumulates_over_micro_batches(dtype, shape, freeze):
+    """Two micro-batches through the same layer: the accumulating backward adds each one's gradients to the buffers
+    (the oracle's two gradients summed in fp64); a frozen factor's buffers keep whatever they held."""
+    M, K, N, r = shape
+    code, tdt = DT[dtype]
+    A = wl.random_factor_case(M, K, N, r, dtype, 8100 + M)
+    Bc = wl.random_factor_case(M + 40, K, N, r, dtype, 8200 + M)
+    Bc["V"], Bc["U"], Bc["b"] = A["V"], A["U"], A["b"]
+    V, U, bias = (dev(A[k], dtype) for k in ("V", "U", "b"))
+    start = {"dU": wl.round_to(wl.normal(8301, (N, r), 0.5), dtype), "dV": wl.round_to(wl.normal(8302, (K, r), 0.5), dtype),
+             "db": wl.round_to(wl.normal(8303, (N,), 0.5), dtype)}
+    dU, dV, db = (dev(start[k], dtype) for k in ("dU", "dV", "db"))
+    want = {k: v.astype(np.float64).copy() for k, v in start.items()}
+    for case in (A, Bc):
+        m = case["M"]
+        desc = b.linear_desc(m, K, N, r, code)
+        ws = workspace(max(b.lrd_linear_workspace_bytes(desc, freeze, 0), b.lrd_linear_workspace_bytes(desc, freeze, 2)))
+        X, dY = dev(case["X"], dtype), dev(case["dY"], dtype)
+        Y = torch.empty(m, N, dtype=tdt, device="cuda")
+        Z = None if freeze == b.LRD_FREEZE_U else torch.empty(m, r, dtype=tdt, device="cuda")
+        dX = torch.empty(m, K, dtype=tdt, device="cuda")
+        b.lrd_linear_fwd(desc, X, V, U, bias, Y, Z, freeze, ws)
+        b.lrd_linear_bwd_accumulate(desc, dY, None if freeze == b.LRD_FREEZE_V else X, V, U, Z, dX, dU, dV, db, freeze, ws)
+        torch.cuda.synchronize()
+        ref = oracle_linear(case, freeze)
+        assert rel_err(dX, ref["dX"]) <= TOL[dtype]
+        for k in want:
+            want[k] += ref[k]                       # zero for a frozen factor
+    assert b.lrd_check_device_status() == b.LRD_OK
+    tol = 2 * TOL[dtype]                            # two roundings to the storage type per accumulation
+    assert rel_err(dU, want["dU"]) <= tol and rel_err(dV, want["dV"]) <= tol and rel_err(db, want["db"]) <= tol
+    if freeze == b.LRD_FREEZE_U:
+        assert np.array_equal(host(dU), start["dU"].astype(np.float64)) and np.array_equal(host(db), start["db"].astype(np.float64))
+    if freeze == b.LRD_FREEZE_V:
+        assert np.array_equal(host(dV), start["dV"].astype(np.float64))

@@ -269,8 +269,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int64_t grow = (int64_t)m0 + row;
             const int64_t gcol0 = (int64_t)n0 + self * cs;
             const uint32_t rot = (uint32_t)row % ngrp;
-            for (uint32_t c4 = 0; c4 < cs; c4 += 8) {
-                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            // 8 columns of this row: the S partials in rank order (+ bias), rounded once
+            auto sum8 = [&](uint32_t c4, uint32_t (&w)[4], float (&acc)[8]) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
                 uint32_t g0 = c4 / 4u + rot, g1 = c4 / 4u + 1u + rot;
                 if (g0 >= ngrp) g0 -= ngrp;
                 if (g1 >= ngrp) g1 -= ngrp;
@@ -284,19 +286,40 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     acc[4] += y.x; acc[5] += y.y; acc[6] += y.z; acc[7] += y.w;
                 }
                 const int64_t col = gcol0 + c4;
-                if (grow < p.M && col < p.N) {
+                if (p.bias) {
+                    for (int e = 0; e < 8; ++e)
+                        if (col + e < p.N) acc[e] += __bfloat162float(p.bias[col + e]);
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) w[e] = pack_bf16(acc[2 * e], acc[2 * e + 1]);
+            };
+            auto store8 = [&](uint32_t c4, const uint32_t (&w)[4], const float (&acc)[8]) {
+                const int64_t col = gcol0 + c4;
+                if (grow >= p.M || col >= p.N) return;
+                __nv_bfloat16* dst = (__nv_bfloat16*)p.C + grow * p.ldc + col;
+                if (col + 8 <= p.N) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+                } else {
+                    for (int e = 0; e < 8; ++e)
+                        if (col + e < p.N) dst[e] = __float2bfloat16_rn(acc[e]);
+                }
+            };
+            // 16 columns (one whole 32-byte sector) per store instruction where the layout allows, else two 16-byte stores
+            const bool sectors = (p.ldc % 16 == 0) && (((uintptr_t)p.C & 31u) == 0) && (gcol0 % 16 == 0);
+            for (uint32_t c4 = 0; c4 < cs; c4 += 16) {
+                uint32_t w0[4], w1[4];
+                float a0[8], a1[8];
+                sum8(c4, w0, a0);
+                const bool second = c4 + 8 < cs;
+                if (second) sum8(c4 + 8, w1, a1);
+                const int64_t col = gcol0 + c4;
+                if (sectors && second && grow < p.M && col + 16 <= p.N) {
                     __nv_bfloat16* dst = (__nv_bfloat16*)p.C + grow * p.ldc + col;
-                    if (p.bias) {
-                        for (int e = 0; e < 8; ++e)
-                            if (col + e < p.N) acc[e] += __bfloat162float(p.bias[col + e]);
-                    }
-                    if (col + 8 <= p.N) {
-                        *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]),
-                                                                    pack_bf16(acc[4], acc[5]), pack_bf16(acc[6], acc[7]));
-                    } else {
-                        for (int e = 0; e < 8; ++e)
-                            if (col + e < p.N) dst[e] = __float2bfloat16_rn(acc[e]);
-                    }
+                    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                 ::"l"(dst), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
+                } else {
+                    store8(c4, w0, a0);
+                    if (second) store8(c4 + 8, w1, a1);
                 }
             }
             if (warp == 2 && lane == 0) { LRD_TS(15); }

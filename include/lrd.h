@@ -132,6 +132,16 @@ lrd_status_t lrd_set_path(lrd_path_t path);
  * thread-safe against concurrent launches.  Returns LRD_ERR_INVALID_ARG for values outside the lists. */
 lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chunk_columns);
 
+/* The fused chain also runs on pairs of SMs (a cluster of 2 S blocks owns 256 rows; the two blocks of a
+ * pair share every MMA and each loads half of the weights): it is taken automatically for layers of more than
+ * 128 rows whose rank splits into S slices of whole 32-column groups.  Overrides for measurement sweeps and
+ * tests (no counterpart in the paper): blocks_per_mma 1 = single-block chain only, 2 = pairs wherever the shape
+ * allows (else the unfused products), 0 = automatic; pairs_per_cluster S (1..4), 64-deep k-blocks per
+ * pipeline stage of the first product (1..4), column-chunk width of the second product (64, 128, 192, 256);
+ * 0 = automatic.  Process-wide, test-only: not thread-safe against concurrent launches.  Returns
+ * LRD_ERR_INVALID_ARG for values outside the lists. */
+lrd_status_t lrd_chain_pair_tuning(int blocks_per_mma, int pairs_per_cluster, int kblocks_per_stage, int chunk_columns);
+
 /* Launch-shape override of the unsplit products (the dense layer's forward and input gradient, the two
  * products of an unfused decomposed layer), for measurement sweeps (no counterpart in the paper):
  * blocks per MMA, 1 (every SM works on its own 128-row tiles) or 2 (pairs of SMs share 256-row tiles and

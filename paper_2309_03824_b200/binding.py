@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
 ]
 
 
@@ -60,6 +60,8 @@ _lib.lrd_rank_search.restype = _i64
 _lib.lrd_rank_search.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double, C.POINTER(C.c_int)]
 _lib.lrd_chain_tuning.restype = _int
 _lib.lrd_chain_tuning.argtypes = [_int, _int, _int]
+_lib.lrd_chain_pair_tuning.restype = _int
+_lib.lrd_chain_pair_tuning.argtypes = [_int, _int, _int, _int]
 _pp = C.POINTER(C.c_void_p)
 _lib.lrd_linear_group_fwd.restype = _int
 _lib.lrd_linear_group_fwd.argtypes = [_int, C.POINTER(lrd_linear_desc_t), _pp, _pp, _pp, _pp, _pp, _pp, _int, _pp,
@@ -173,6 +175,10 @@ def lrd_set_path(path):
 
 def lrd_chain_tuning(cluster_blocks=0, kblocks_per_stage=0, chunk_columns=0):
     _check(_lib.lrd_chain_tuning(cluster_blocks, kblocks_per_stage, chunk_columns))
+
+
+def lrd_chain_pair_tuning(blocks_per_mma=0, pairs_per_cluster=0, kblocks_per_stage=0, chunk_columns=0):
+    _check(_lib.lrd_chain_pair_tuning(blocks_per_mma, pairs_per_cluster, kblocks_per_stage, chunk_columns))
 
 
 def lrd_gemm_tuning(blocks_per_mma=0):

@@ -25,10 +25,6 @@
 #include "tc.cuh"
 #include "tma.cuh"
 
-#ifndef LRD_TS
-#define LRD_TS(slot)      // timestamp hook of profiling builds (one thread, clock counter into a trace buffer); compiled out
-#endif
-
 namespace lrd {
 namespace {
 
@@ -68,11 +64,14 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    // phase 1: [T | ring of S1 stages];  phase 2: [T | two output slabs | ring of S2 stages]
+    // phase 1: [ring of S1 stages] over ALL of the shared memory (T is written only after the last MMA of phase 1 has
+    // read its operands);  afterwards: [T | output slabs | ring of S2 stages].  What a block can stream is (bytes of
+    // stages in flight) / (about a microsecond per stage turn: load latency under load, then its MMAs), so phase 1
+    // gets every byte there is.
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t t_base = smem_base;
-    const uint32_t ring1_base = t_base + p.t_bytes;
-    const uint32_t staging_base = ring1_base;
+    const uint32_t ring1_base = smem_base;
+    const uint32_t staging_base = t_base + p.t_bytes;
     const uint32_t ring2_base = staging_base + kStagingBytes;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
     const uint32_t t_sw = 2u * (uint32_t)p.taw, t_atom_bytes = 128u * t_sw;   // T: atoms of [128 rows x taw columns]
@@ -98,7 +97,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         fence_mbar_init();
     }
     if (threadIdx.x == 0) {
-        LRD_TS(0);
         abort_flag = 0;
         prefetch_tmap(&tmIn);
         prefetch_tmap(&tmP);
@@ -122,16 +120,16 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     }
     tc_fence_before();
     __syncthreads();
-    // Cluster barrier 1 (every block's barriers exist before a peer pushes into it): arrive now, wait
-    // only where the first remote operation is near.  Until then a block touches its own memory only.
-    cluster_arrive();
+    // Cluster barrier 1 (every block's barriers exist, and its phase-1 ring -- which covers the region the peers'
+    // slices of T land in -- is dead, before a peer pushes into it): the gather warps arrive once this block's
+    // phase-1 MMAs have completed, the other warps now; waited on only where the first remote operation is near.
+    if (warp < 2) cluster_arrive();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     // Everything above touched only this block's own shared and tensor memory, so it may overlap the tail
     // of the previous kernel in the stream; global memory is first read (and written) below this line.
     griddep_launch_dependents();
     griddep_wait();
-    if (threadIdx.x == 0) { LRD_TS(1); }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -147,7 +145,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             const uint32_t dst = ring1_base + s * p.stage1_bytes;
             const int kb0 = g * p.G1;
             if (elect_one()) {
-                if (g == 0) { LRD_TS(2); }
                 mbar_expect_tx(fb, p.stage1_bytes);
                 for (int i = 0; i < p.G1; ++i)               // k-blocks past K1 read as zeros
                     tma_load_2d(dst + i * kInTileBytes, &tmIn, fb, (kb0 + i) * 64, m0);
@@ -157,10 +154,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             __syncwarp();
             if (++s == p.S1) { s = 0; ph ^= 1; }
         }
-        if (lane == 0) { LRD_TS(3); }
         // the ring is laid out anew for phase 2: wait until every phase-1 MMA has read its operands
         if (ok) ok = mbar_wait_uniform(smem_u32(&tacc_bar), 0, ab);
-        if (lane == 0) { LRD_TS(4); }
         s = 0;
         ph = 1;
         for (int j = c; j < p.n_chunks && ok; j += p.C) {
@@ -177,7 +172,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 if (++s == p.S2) { s = 0; ph ^= 1; }
             }
         }
-        if (lane == 0) { LRD_TS(5); }
         cluster_wait();        // barrier 1
         cluster_arrive_relaxed();   // barrier 2 (progress only)
     } else if (warp == 1) {
@@ -191,7 +185,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         for (int g = 0; g < ng1; ++g) {
             ok = mbar_wait_uniform(smem_u32(&full1[s]), ph, ab);
             if (!ok) break;
-            if (g == 0 && lane == 0) { LRD_TS(6); }
             tc_fence_after();
             const uint32_t in_src = ring1_base + s * p.stage1_bytes;
             const uint32_t p_src = in_src + p.G1 * kInTileBytes;
@@ -214,13 +207,11 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         }
         if (ok && elect_one()) mma_commit(smem_u32(&tacc_bar));
         __syncwarp();
-        if (lane == 0) { LRD_TS(7); }
         // this block's own slice is in its T buffer, which also means that the phase-1 accumulator columns
         // (which the first chunk's accumulator overlaps) have been read out; the peers' slices are waited for
         // where the k-loop first touches them
         if (ok) ok = mbar_wait_uniform(smem_u32(&tready_bar[c]), 0, ab);
         uint32_t slices_ready = 1u << c;
-        if (lane == 0) { LRD_TS(8); }
         const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
         const uint64_t t_desc0 = smem_desc(t_base, 0, 8u * t_sw, t_sw);
         s = 0;
@@ -244,7 +235,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 }
                 ok = mbar_wait_uniform(smem_u32(&full2[s]), ph, ab);
                 if (!ok) break;
-                if (i2 == 0 && i < 8 && lane == 0) { LRD_TS(24 + i); }
                 tc_fence_after();
                 const uint32_t q_src = ring2_base + s * p.stage2_bytes;
                 const uint64_t bd = a_desc0 + ((q_src >> 4) & 0x3FFFu);
@@ -258,11 +248,9 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                     if (i == p.kb2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
                 }
                 __syncwarp();
-                if (i2 == 0 && i < 8 && lane == 0) { LRD_TS(32 + i); }
                 if (++s == p.S2) { s = 0; ph ^= 1; }
             }
         }
-        if (lane == 0) { LRD_TS(9); }
         // a block without a chunk of its own still has to have received every slice before it passes barrier 2
         for (int j = 0; j < p.C && ok; ++j)
             if (!((slices_ready >> j) & 1u)) ok = mbar_wait_cluster_uniform(smem_u32(&tready_bar[j]), 0, ab);
@@ -277,7 +265,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         bool ok = mbar_wait_uniform(smem_u32(&tacc_bar), 0, ab);   // warp-uniform from here on
         tc_fence_after();
-        if (lead_warp && lane == 0) { LRD_TS(10); }
+        cluster_arrive_relaxed();   // barrier 1: this block's phase-1 ring is dead (progress only, no data)
         if (ok) {
             // 32 columns per step (two tensor-memory loads in flight, one wait), a 16-column tail if RS / 16 is odd
             for (int col = 0; col < p.RS; col += 32) {
@@ -306,14 +294,12 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         // the four warps have written it, one thread copies it into every peer's buffer (bulk DSMEM copy that
         // completes on the peer's barrier) and, if asked, stores it to T_save.  The accumulator columns of
         // the slice are free for phase 2 from here on.
-        if (lead_warp && lane == 0) { LRD_TS(17); }
         fence_proxy_async_smem();
         tc_fence_before();
         cluster_wait();        // barrier 1: the peers' barriers exist
         named_bar_sync(2, 128);
         if (lead_warp) {
             if (ok && elect_one()) {
-                LRD_TS(11);
                 const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;
                 for (int t = 1; t < p.C; ++t) {
                     const uint32_t peer = (uint32_t)((c + t) % p.C);
@@ -325,7 +311,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                         tma_store_2d(&tmT, slice + (uint32_t)a * t_atom_bytes, c * p.RS + a * p.taw, m0);
                     tma_store_commit();
                 }
-                LRD_TS(12);
             }
             __syncwarp();
         }
@@ -349,7 +334,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             ok = named_bar_and(3, 128, ok);                  // the four warps go on, or give up, together (and see the bias)
             if (!ok) break;
             if (!arrived2) { cluster_arrive_relaxed(); arrived2 = true; }   // barrier 2 (T was complete before these MMAs)
-            if (lead_warp && lane == 0 && i == 0) { LRD_TS(13); }
             tc_fence_after();
             const uint32_t d_tmem = lane_addr + (uint32_t)buf * 256u;
             for (int g = 0; g * 64 < p.BN2; ++g) {
@@ -358,7 +342,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 uint32_t v[64];                              // both halves are loaded before the first is converted
                 tmem_ld_32x32(d_tmem + g * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
                 tmem_ld_32x32(d_tmem + g * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-                if (lead_warp && lane == 0 && sb < 8) { LRD_TS(40 + 2 * sb); }
                 tmem_ld_wait();
 #pragma unroll
                 for (int h = 0; h < 2; ++h, ++sb) {
@@ -394,16 +377,13 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                     }
                     __syncwarp();
                 }
-                if (lead_warp && lane == 0 && sb <= 8) { LRD_TS(41 + 2 * (sb - 2)); }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&out_empty[buf]));
         }
         if (!arrived2) cluster_arrive_relaxed();
-        if (lead_warp && lane == 0) { LRD_TS(14); }
         tma_store_wait_read<0>();                            // shared memory may go once the stores have read it
-        if (lead_warp && lane == 0) { LRD_TS(15); }
         __syncwarp();
     }
 
@@ -412,7 +392,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     cluster_wait();
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) { LRD_TS(16); }
     if (warp == 1) {
         if (abort_flag) {
             for (int i = 0; i < 256; ++i) __nanosleep(1000);
@@ -494,8 +473,8 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         if (RS > 256) continue;
         const int swb = RS % 64 == 0 ? 128 : (RS % 32 == 0 ? 64 : 32);
         const int BN2 = pick_bn2(a.N2, C);
-        const int64_t ring1 = (int64_t)kSmemLimit - 1024 - t_bytes;
-        const int64_t ring2 = ring1 - (int64_t)kStagingBytes;
+        const int64_t ring1 = (int64_t)kSmemLimit - 1024;                         // phase 1 has all of it
+        const int64_t ring2 = ring1 - t_bytes - (int64_t)kStagingBytes;
         const uint32_t kb1_bytes = kInTileBytes + 128u * RS, kb2_bytes = (uint32_t)BN2 * 128u;
         if (ring2 < 2 * (int64_t)kb2_bytes) continue;
         // phase 1: one k-block per stage (the finest pipeline); two for a short reduction, where the number of
@@ -510,7 +489,8 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         if (S2 > kMaxStages) S2 = kMaxStages;
         const uint32_t s1b = (uint32_t)G1 * kb1_bytes;
         const uint32_t used1 = (uint32_t)S1 * s1b, used2 = kStagingBytes + (uint32_t)S2 * kb2_bytes;
-        Plan pl{C, RS, swb, BN2, G1, S1, S2, s1b, kb2_bytes, (uint32_t)t_bytes, 1024u + (uint32_t)t_bytes + (used1 > used2 ? used1 : used2)};
+        const uint32_t after1 = (uint32_t)t_bytes + used2;
+        Plan pl{C, RS, swb, BN2, G1, S1, S2, s1b, kb2_bytes, (uint32_t)t_bytes, 1024u + (used1 > after1 ? used1 : after1)};
         // prefer the largest cluster whose blocks are all resident at once (within this launch's share of the
         // SMs, when it runs beside other launches); else the smallest feasible
         if (!found) { best = pl; found = true; }
@@ -537,13 +517,13 @@ bool chain_eligible(const ChainArgs& a) {
 }
 
 // The fused kernel loses to two separate products where the T buffer (128 rows x r) leaves room for only two
-// k-blocks of phase 1 in flight, i.e. at r = 512 (measured at 8192 tokens: 1024 -> 4096 forward 65 us fused against 49 us on two
+// Q tiles of phase 2 in flight, i.e. at r = 512 (measured at 8192 tokens: 1024 -> 4096 forward 65 us fused against 49 us on two
 // persistent products, 4096 -> 1024 99 against 46 us; at r <= 384 the chain wins everywhere measured).  The
 // automatic path then takes the separate products; LRD_PATH_FUSED still forces the chain.
 bool chain_preferred(const ChainArgs& a) {
     Plan pl;
     if (!make_plan(a, &pl)) return false;
-    return pl.S1 * pl.G1 > 2;          // k-blocks of phase 1 in flight
+    return pl.S2 >= 3;                 // Q tiles of phase 2 in flight
 }
 
 lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {

@@ -27,4 +27,14 @@ bool chain_eligible(const ChainArgs& c);
 bool chain_preferred(const ChainArgs& c);
 lrd_status_t chain_launch(const ChainArgs& c, cudaStream_t stream);
 
+// The same chain on pairs of SMs (tcgen05 cta_group::2): a cluster of 2 S blocks owns 256 rows.  `layers` are
+// n <= kChainMaxLayers independent layers of equal shape that run in one launch (gridDim.z).  Needs more than
+// 128 rows and a rank that splits into S slices of whole 32-column groups.
+constexpr int kChainMaxLayers = 4;
+// Overrides for sweeps and tests: pairs per cluster (1-4), k-blocks per phase-1 stage, phase-2 chunk width; 0 = automatic.
+void chain_pair_tuning(int S, int G1, int BN2);
+bool chain_pair_eligible(const ChainArgs* layers, int n);
+bool chain_pair_preferred(const ChainArgs* layers, int n);
+lrd_status_t chain_pair_launch(const ChainArgs* layers, int n, cudaStream_t stream);
+
 }  // namespace lrd

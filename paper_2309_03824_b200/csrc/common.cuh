@@ -27,6 +27,10 @@ struct GemmArgs {
     lrd_dtype_t dtype;         // storage type of A, B, C, bias
 };
 
+// True when the CUDA call succeeded.  With the environment variable LRD_LOG_ERRORS set, a failure is also written to
+// stderr with the call's name and CUDA's error string (the C ABI itself only returns LRD_ERR_CUDA).
+bool cuda_ok(cudaError_t e, const char* what);
+
 // Host-side count of kernels enqueued (see lrd_launch_count).
 void count_launch(int n = 1);
 

@@ -4,6 +4,8 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cstdio>
+#include <cstdlib>
 
 #include "chain.cuh"
 #include "common.cuh"
@@ -16,6 +18,7 @@ using namespace lrd;
 namespace {
 
 std::atomic<int> g_path{LRD_PATH_AUTO};
+std::atomic<int> g_chain_mma_blocks{0};     // 0: automatic; 1: single-block chain only; 2: the chain on pairs of SMs wherever it is eligible
 std::atomic<uint64_t> g_launches{0};
 
 lrd_status_t check_arch() {
@@ -71,6 +74,38 @@ GemmArgs gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool 
     return make_gemm(M, N, K, A, lda, a_mn, B, ldb, b_mn, C, ldc, bias, dt);
 }
 
+// The fused chain for one layer, or for n layers of equal shape in one launch: on pairs of SMs where the shape
+// allows, else (one layer only) on single blocks.  Returns LRD_ERR_UNSUPPORTED when no fused kernel takes it.
+lrd_status_t launch_chain(const ChainArgs* c, int n, int path, cudaStream_t s) {
+    const int mode = g_chain_mma_blocks.load();
+    const bool forced = path == LRD_PATH_FUSED;
+    if (c[0].sm_share == 0 && mode != 1) {
+        if (mode == 2 || forced ? chain_pair_eligible(c, n) : chain_pair_preferred(c, n)) return chain_pair_launch(c, n, s);
+    }
+    if (n != 1 || mode == 2) return LRD_ERR_UNSUPPORTED;
+    if (forced ? chain_eligible(c[0]) : chain_preferred(c[0])) return chain_launch(c[0], s);
+    return LRD_ERR_UNSUPPORTED;
+}
+
+ChainArgs fwd_chain_args(const Linear& L, const void* X, const void* V, const void* U, const void* bias, void* Y, void* Z_save,
+                         int sm_share) {
+    ChainArgs c;
+    c.M = L.M; c.K1 = L.K; c.r = L.r; c.N2 = L.N;
+    c.In = X; c.ld_in = L.ldx; c.P = V; c.ldp = L.ldv; c.Q = U; c.ldq = L.ldu; c.bias = bias;
+    c.Out = Y; c.ld_out = L.ldy; c.T_save = Z_save; c.ldt = L.ldz; c.dtype = L.dt;
+    c.sm_share = sm_share;
+    return c;
+}
+
+ChainArgs bwd_chain_args(const Linear& L, const void* dY, const void* V, const void* U, void* dX, void* dZ_save, int sm_share) {
+    ChainArgs c;
+    c.M = L.M; c.K1 = L.N; c.r = L.r; c.N2 = L.K;
+    c.In = dY; c.ld_in = L.ldy; c.P = U; c.ldp = L.ldu; c.Q = V; c.ldq = L.ldv; c.bias = nullptr;
+    c.Out = dX; c.ld_out = L.ldx; c.T_save = dZ_save; c.ldt = L.r; c.dtype = L.dt;
+    c.sm_share = sm_share;
+    return c;
+}
+
 size_t linear_z_bytes(const Linear& L) { return align_up((size_t)(L.M > 0 ? L.M : 1) * L.r * elem_size(L.dt), 256); }
 
 size_t linear_grad_scratch_bytes(const Linear& L) {     // dU, dV and dbias of one step, in the parameters' layouts
@@ -100,6 +135,13 @@ size_t linear_split_bytes(const Linear& L) {     // scratch after dZ: split part
 namespace lrd {
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n); }
+
+bool cuda_ok(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return true;
+    static const bool log = getenv("LRD_LOG_ERRORS") != nullptr;
+    if (log) fprintf(stderr, "lrd: %s failed: %s\n", what, cudaGetErrorString(e));
+    return false;
+}
 
 lrd_status_t run_gemm(const GemmArgs& g, int path, bool allow_split, float* partials, size_t partial_bytes,
                       cudaStream_t s) {
@@ -239,6 +281,16 @@ lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chu
     return LRD_OK;
 }
 
+lrd_status_t lrd_chain_pair_tuning(int blocks_per_mma, int pairs_per_cluster, int kblocks_per_stage, int chunk_columns) {
+    if (blocks_per_mma < 0 || blocks_per_mma > 2) return LRD_ERR_INVALID_ARG;
+    if (pairs_per_cluster < 0 || pairs_per_cluster > 4) return LRD_ERR_INVALID_ARG;
+    if (kblocks_per_stage < 0 || kblocks_per_stage > 4) return LRD_ERR_INVALID_ARG;
+    if (chunk_columns != 0 && chunk_columns != 64 && chunk_columns != 128 && chunk_columns != 192 && chunk_columns != 256) return LRD_ERR_INVALID_ARG;
+    g_chain_mma_blocks.store(blocks_per_mma);
+    chain_pair_tuning(pairs_per_cluster, kblocks_per_stage, chunk_columns);
+    return LRD_OK;
+}
+
 lrd_status_t lrd_gemm_tuning(int blocks_per_mma) {
     if (blocks_per_mma < 0 || blocks_per_mma > 2) return LRD_ERR_INVALID_ARG;
     tc_gemm_persistent_force_pairs(blocks_per_mma);
@@ -297,12 +349,9 @@ static lrd_status_t linear_fwd_on(const lrd_linear_desc_t* desc, const void* X, 
 
     const int path = g_path.load();
     if (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) {
-        ChainArgs c;
-        c.M = L.M; c.K1 = L.K; c.r = L.r; c.N2 = L.N;
-        c.In = X; c.ld_in = L.ldx; c.P = V; c.ldp = L.ldv; c.Q = U; c.ldq = L.ldu; c.bias = bias;
-        c.Out = Y; c.ld_out = L.ldy; c.T_save = Z_save; c.ldt = L.ldz; c.dtype = L.dt;
-        c.sm_share = sm_share;
-        if (path == LRD_PATH_FUSED ? chain_eligible(c) : chain_preferred(c)) return chain_launch(c, s);
+        const ChainArgs c = fwd_chain_args(L, X, V, U, bias, Y, Z_save, sm_share);
+        const lrd_status_t st = launch_chain(&c, 1, path, s);
+        if (st != LRD_ERR_UNSUPPORTED) return st;
     }
     void* Z = Z_save ? Z_save : workspace;
     const int64_t ldz = Z_save ? L.ldz : L.r;
@@ -323,7 +372,8 @@ lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const 
 static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
                                   const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                                   lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, cudaStream_t s,
-                                  cudaStream_t side, cudaEvent_t side_done, int sm_share, bool check_only = false) {
+                                  cudaStream_t side, cudaEvent_t side_done, int sm_share, bool check_only = false,
+                                  bool data_done = false) {
     Linear L;
     LRD_TRY(parse_linear(desc, &L, false));
     const uint32_t plan = lrd_linear_bwd_plan(freeze);
@@ -355,18 +405,13 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
     const size_t partial_bytes = workspace_bytes - linear_z_bytes(L);
     const bool need_dz_in_memory = (plan & LRD_PLAN_DV) != 0;
 
-    bool chained = false;
+    bool chained = data_done;            // a group has already run this layer's data chain (dX, and dZ where needed)
     const int path = g_path.load();
-    if (dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED)) {
-        ChainArgs c;
-        c.M = L.M; c.K1 = L.N; c.r = L.r; c.N2 = L.K;
-        c.In = dY; c.ld_in = L.ldy; c.P = U; c.ldp = L.ldu; c.Q = V; c.ldq = L.ldv; c.bias = nullptr;
-        c.Out = dX; c.ld_out = L.ldx; c.T_save = need_dz_in_memory ? dZ : nullptr; c.ldt = L.r; c.dtype = L.dt;
-        c.sm_share = sm_share;
-        if (path == LRD_PATH_FUSED ? chain_eligible(c) : chain_preferred(c)) {
-            LRD_TRY(chain_launch(c, s));
-            chained = true;
-        }
+    if (!chained && dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED)) {
+        const ChainArgs c = bwd_chain_args(L, dY, V, U, dX, need_dz_in_memory ? dZ : nullptr, sm_share);
+        const lrd_status_t st = launch_chain(&c, 1, path, s);
+        if (st == LRD_OK) chained = true;
+        else if (st != LRD_ERR_UNSUPPORTED) return st;
     }
     if (!chained) {
         if (dX || need_dz_in_memory)
@@ -448,6 +493,18 @@ lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const v
     for (int i = 0; i < n; ++i)          // nothing is enqueued unless every layer's arguments are valid
         LRD_TRY(linear_fwd_on(&descs[i], X[i], V[i], U[i], bias ? bias[i] : nullptr, Y[i], Z_save ? Z_save[i] : nullptr, freeze,
                               workspace[i], workspace_bytes[i], s, 0, true));
+    // layers of one shape: one launch of the fused chain on pairs of SMs, the layer picked by gridDim.z
+    const int path = g_path.load();
+    if (n > 1 && n <= kChainMaxLayers && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) && g_chain_mma_blocks.load() != 1) {
+        ChainArgs c[kChainMaxLayers];
+        bool ok = true;
+        for (int i = 0; i < n && ok; ++i) {
+            Linear L;
+            ok = parse_linear(&descs[i], &L, false) == LRD_OK && L.M > 0;
+            if (ok) c[i] = fwd_chain_args(L, X[i], V[i], U[i], bias ? bias[i] : nullptr, Y[i], Z_save ? Z_save[i] : nullptr, 0);
+        }
+        if (ok && chain_pair_eligible(c, n)) return chain_pair_launch(c, n, s);
+    }
     SideStreams* ss = n > 1 ? side_streams() : nullptr;
     if (n > 1 && !ss) return LRD_ERR_CUDA;
     if (n > 1 && cudaEventRecord(ss->fork, s) != cudaSuccess) return LRD_ERR_CUDA;
@@ -481,6 +538,25 @@ lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const v
     if (!ss) return LRD_ERR_CUDA;
     if (cudaEventRecord(ss->fork, s) != cudaSuccess) return LRD_ERR_CUDA;
     const bool du_aside = (lrd_linear_bwd_plan(freeze) & LRD_PLAN_DU) != 0;
+    // layers of one shape: their data chains (dZ, dX) in one launch on pairs of SMs, the layer picked by gridDim.z;
+    // the weight gradients then run side by side as below
+    bool data_done = false;
+    const int path = g_path.load();
+    if (n > 1 && n <= kChainMaxLayers && dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) && g_chain_mma_blocks.load() != 1) {
+        ChainArgs c[kChainMaxLayers];
+        bool ok = true;
+        const bool need_dz = (lrd_linear_bwd_plan(freeze) & LRD_PLAN_DV) != 0;
+        for (int i = 0; i < n && ok; ++i) {
+            Linear L;
+            ok = parse_linear(&descs[i], &L, false) == LRD_OK && L.M > 0 && dX[i] != nullptr;
+            if (ok) c[i] = bwd_chain_args(L, dY[i], V[i], U[i], dX[i], need_dz ? workspace[i] : nullptr, 0);
+        }
+        if (ok && chain_pair_eligible(c, n)) {
+            LRD_TRY(chain_pair_launch(c, n, s));
+            data_done = true;
+            if (!cuda_ok(cudaEventRecord(ss->mid, s), "cudaEventRecord(group mid)")) return LRD_ERR_CUDA;
+        }
+    }
     // The data chains are shaped for twice their even share: the weight-gradient launches that follow each of them
     // fill the machine anyway, and a chain of 2 blocks per row tile finishes sooner than one of 1 (three
     // 768 -> 768, r = 192 layers at 4096 tokens, U frozen: 32.9 us against 35.3 us).
@@ -489,11 +565,11 @@ lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const v
     for (int i = 0; i < n; ++i) {
         cudaStream_t si = i == 0 ? s : ss->layer[i - 1];
         cudaStream_t sd = du_aside ? ss->aux[i] : nullptr;
-        if (i > 0 && cudaStreamWaitEvent(si, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
+        if (i > 0 && !cuda_ok(cudaStreamWaitEvent(si, data_done ? ss->mid : ss->fork, 0), "cudaStreamWaitEvent(group layer)")) { st = LRD_ERR_CUDA; continue; }
         if (sd && cudaStreamWaitEvent(sd, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
         const lrd_status_t sti = linear_bwd_on(&descs[i], dY[i], at(X, i), V[i], U[i], at(Z_save, i), at_w(dX, i), at_w(dU, i),
                                                at_w(dV, i), at_w(dbias, i), freeze, workspace[i], workspace_bytes[i], si, sd,
-                                               ss->aux_done[i], share);
+                                               ss->aux_done[i], share, false, data_done);
         if (sti != LRD_OK) st = sti;
         if (sd && !stream_after(s, sd, ss->aux_done[i])) st = LRD_ERR_CUDA;
         if (i > 0 && !stream_after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;

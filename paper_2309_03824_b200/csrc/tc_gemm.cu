@@ -23,10 +23,6 @@
 #include "tc.cuh"
 #include "tma.cuh"
 
-#ifndef LRD_TS
-#define LRD_TS(slot)      // timestamp hook of profiling builds; compiled out
-#endif
-
 namespace lrd {
 namespace {
 
@@ -85,7 +81,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int kb_end = min(kb_begin + p.kb_per_split, p.kb_total);
 
     if (threadIdx.x == 0) {
-        LRD_TS(0);
         abort_flag = 0;
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
@@ -121,7 +116,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // previous kernel in the stream; global memory is first touched below this line
     griddep_launch_dependents();
     griddep_wait();
-    if (threadIdx.x == 0) { LRD_TS(1); }
 
     if (warp == 0) {
         // TMA producer: the whole warp runs the loop, one elected lane issues (operands stay uniform)
@@ -135,7 +129,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t b_dst = a_dst + A_STAGE_BYTES;
             const int k0 = kb * BK;
             if (elect_one()) {
-                if (it == 0) { LRD_TS(2); }
                 mbar_expect_tx(fb, A_STAGE_BYTES + BN * BK * 2);
                 if (A_MN) {
 #pragma unroll
@@ -152,7 +145,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             __syncwarp();
         }
-        if (lane == 0) { LRD_TS(3); }
         if (p.cluster_splits > 1) { cluster_arrive(); cluster_wait(); cluster_arrive_relaxed(); }   // barriers 1 and 2, see the epilogue
     } else if (warp == 1) {
         // MMA issuer: converged warp, elect.sync around the issue
@@ -163,7 +155,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = kb_begin; kb < kb_end; ++kb) {
             ok = mbar_wait_uniform(smem_u32(&full_bar[s]), ph, ab);
             if (!ok) break;
-            if (kb == kb_begin && lane == 0) { LRD_TS(4); }
             tc_fence_after();
             const uint32_t a_src = smem_base + s * C::STAGE_BYTES;
             const uint32_t b_src = a_src + A_STAGE_BYTES;
@@ -183,7 +174,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (ok && elect_one()) mma_commit(smem_u32(&acc_bar));
         __syncwarp();
-        if (lane == 0) { LRD_TS(5); }
         if (p.cluster_splits > 1) { cluster_arrive(); cluster_wait(); cluster_arrive_relaxed(); }
     } else if (p.cluster_splits > 1) {
         // ---- cluster split: reduce the partial tiles of the cluster's blocks through shared memory ----
@@ -197,11 +187,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool with_colsum = ONES && blockIdx.x == 0;
         bool ok = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
         tc_fence_after();
-        if (warp == 2 && lane == 0) { LRD_TS(6); }
         // barrier 1: this block's pipeline ring is dead (all its MMAs have completed).  Progress only: what the peers
         // must see of this block (its initialised barriers) is released by the arrivals of warps 0 and 1.
         cluster_arrive_relaxed();
-        if (warp == 2 && lane == 0) { LRD_TS(13); }
         if (ok) {
             // partial tile -> staging, laid out [owner][row][cs] so that each owner's slice is one contiguous range
             const bool has_work = kb_begin < kb_end;       // a block past the end of the reduction contributes zeros
@@ -238,12 +226,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 asm volatile("st.shared.u32 [%0], %1;" ::"r"(cs_stage + (uint32_t)row * 4u), "r"(cv[0]) : "memory");
             }
         }
-        if (warp == 2 && lane == 0) { LRD_TS(7); }
         fence_proxy_async_smem();
         tc_fence_before();
         cluster_wait();        // barrier 1 complete: every peer's ring is dead, its receive slots may be written
         ok = named_bar_and(2, 128, ok);
-        if (warp == 2 && lane == 0) { LRD_TS(8); }
         if (warp == 2) {
             if (ok && elect_one()) {
                 for (uint32_t t = 1; t < S; ++t) {
@@ -254,16 +240,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             __syncwarp();
         }
-        if (warp == 2 && lane == 0) { LRD_TS(9); }
         if (ok) {
             bool got = false;
             if (lane == 0) got = mbar_wait_cluster(smem_u32(&red_bar), 0, ab);
             ok = __shfl_sync(0xffffffffu, got ? 1 : 0, 0) != 0;
             if (ok) { for (int i = 0; i < 64 && !mbar_try_wait_cluster(smem_u32(&red_bar), 0); ++i) {} }
         }
-        if (warp == 2 && lane == 0) { LRD_TS(10); }
         cluster_arrive_relaxed();   // barrier 2: everything addressed to this block has landed (progress only, no data)
-        if (warp == 2 && lane == 0) { LRD_TS(14); }
         if (ok) {
             // this block's column slice: add the S partials in rank order, round once, store
             const int64_t grow = (int64_t)m0 + row;
@@ -322,7 +305,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (second) store8(c4 + 8, w1, a1);
                 }
             }
-            if (warp == 2 && lane == 0) { LRD_TS(15); }
             if (with_colsum && self == 0 && p.colsum_out && grow < p.M) {
                 float t = 0.f;
                 for (uint32_t k = 0; k < S; ++k) {
@@ -334,7 +316,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 p.colsum_out[grow] = __float2bfloat16_rn(t);
             }
         }
-        if (warp == 2 && lane == 0) { LRD_TS(11); }
     } else {
         const int quarter = warp % 4;                      // lanes [32 q, 32 q + 32) of tensor memory
         const bool ready = mbar_wait_warp(smem_u32(&acc_bar), 0, ab);
@@ -409,7 +390,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (p.cluster_splits > 1) cluster_wait();
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) { LRD_TS(12); }
     if (warp == 1) {
         if (abort_flag) {            // give copies and MMAs still in flight time to land before freeing
             for (int i = 0; i < 256; ++i) __nanosleep(1000);

@@ -1,5 +1,7 @@
 #include "tma.cuh"
 
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 namespace lrd {
@@ -35,9 +37,19 @@ bool make_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64
     const CUtensorMapSwizzle sw = box_cols * 2 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                  : box_cols * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
                                  : box_cols * 2 == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
-    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc == CUDA_ERROR_INVALID_CONTEXT) {
+        // a host thread whose first CUDA work is this call has no context bound yet: the driver's encoder wants one,
+        // any runtime call that touches the device binds the primary context
+        cudaFree(nullptr);
+        rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (rc != CUDA_SUCCESS && getenv("LRD_LOG_ERRORS"))
+        fprintf(stderr, "lrd: cuTensorMapEncodeTiled failed (%d): base %p rows %llu cols %llu ld %llu box %u x %u\n", (int)rc, base,
+                (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)ld_elems, box_rows, box_cols);
+    return rc == CUDA_SUCCESS;
 }
 
 bool make_tmap_nhwc_bf16(CUtensorMap* out, const void* base, uint64_t B, uint64_t H, uint64_t W, uint64_t C,

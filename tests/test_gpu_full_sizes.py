@@ -47,6 +47,16 @@ def test_rank_sweep_layer_full_size(r, freeze):
     check_sampled(wl.random_factor_case(c["M"], c["K"], c["N"], r, "bf16", 2000 + r), freeze)
 
 
+@pytest.mark.parametrize("r", [100, 250, 500, 750, 1000, 504, 752])
+@pytest.mark.parametrize("freeze", [b.LRD_FREEZE_NONE, b.LRD_FREEZE_V])
+def test_rank_sweep_packed_and_rounded_to_8_full_size(r, freeze):
+    """The sweep's unquantized ranks stored packed (leading dimension = r: rows of V, U, Z, dU, dV start at
+    addresses that are not multiples of 16 bytes) and the ranks rounded up to a multiple of 8 that are not
+    multiples of 16, under both masks the workload names."""
+    c = wl.C2_SWEEP
+    check_sampled(wl.random_factor_case(c["M"], c["K"], c["N"], r, "bf16", 2100 + r), freeze)
+
+
 @pytest.mark.parametrize("layer", wl.C4_GPT_LAYERS[3:], ids=[l[0] for l in wl.C4_GPT_LAYERS[3:]])
 @pytest.mark.parametrize("freeze", [b.LRD_FREEZE_U, b.LRD_FREEZE_V])
 def test_gpt2_medium_shaped_layers_full_size(layer, freeze):

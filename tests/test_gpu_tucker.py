@@ -73,6 +73,16 @@ def test_tensor_core_path(geom, freeze):
     check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 500 + C), freeze)
 
 
+@pytest.mark.parametrize("geom", [(2, 7, 7, 512, 512, 136, 136), (2, 7, 7, 512, 512, 256, 256), (1, 7, 7, 512, 512, 304, 248),
+                                  (3, 7, 7, 512, 512, 312, 312)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_tensor_core_path_ranks_above_128(geom, freeze):
+    """The [512, 512, 3, 3] layer on 7 x 7 images at ranks between Eq. 6's and Eq. 5's: several 128-column output
+    tiles of the core and three to five 64-channel blocks per filter tap."""
+    B, H, W, C, S, r1, r2 = geom
+    check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 700 + r1), freeze)
+
+
 @pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 5, 7, 12, 10, 5, 6)])
 @pytest.mark.parametrize("freeze", MASKS)
 def test_backward_launches_side_by_side_or_in_a_row_give_the_same_bits(geom, freeze):

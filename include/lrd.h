@@ -26,7 +26,10 @@
  *    out raises a device-side flag that lrd_check_device_status() reports as LRD_ERR_TIMEOUT.
  *  - Ranks and sizes that do not meet the alignment needs of the tensor-core path (every
  *    leading dimension a multiple of 8 elements and every base pointer 16-byte aligned, bf16)
- *    are supported through a slower general path; they are not errors.
+ *    are supported, not errors.  A bf16 layer whose FACTORS are stored with other leading dimensions
+ *    (an unquantized rank stored packed) still runs on the tensor cores: its factors are copied into
+ *    the workspace with padded rows (lrd_linear_workspace_bytes accounts for it).  Activations with
+ *    such leading dimensions, bases off a 16-byte boundary and fp32 take a slower general path.
  *  - Devices other than compute capability 10.x return LRD_ERR_ARCH.  There is no CPU path.
  */
 #ifndef LRD_H_
@@ -161,6 +164,14 @@ lrd_status_t lrd_tucker2_overlap(int on);
 /* Synchronises the current device, then reports and clears the device-side timeout flag:
  * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
 lrd_status_t lrd_check_device_status(void);
+
+/* Self-test of the bounded device-side wait (no counterpart in the paper): enqueues one small block that waits,
+ * through the same routine and with the same limit as every pipeline wait of the library's kernels, on a barrier
+ * nothing ever arrives at.  The wait runs out after a second or so, raises the timeout flag and the block
+ * returns in order (nothing is in flight, no tensor memory is held).  The next lrd_check_device_status() returns
+ * LRD_ERR_TIMEOUT once, the one after LRD_OK, and every other entry point keeps working.  Returns
+ * LRD_ERR_ARCH / LRD_ERR_CUDA as the other entry points do. */
+lrd_status_t lrd_selftest_wait_timeout(void* cuda_stream);
 
 /* Number of kernels this library has enqueued since it was loaded (host-side counter, all
  * streams; memset nodes of zero-filled gradients are not counted).  For launch accounting. */

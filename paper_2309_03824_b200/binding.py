@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_selftest_wait_timeout", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
 ]
 
 
@@ -60,6 +60,8 @@ _lib.lrd_rank_search.restype = _i64
 _lib.lrd_rank_search.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double, C.POINTER(C.c_int)]
 _lib.lrd_chain_tuning.restype = _int
 _lib.lrd_chain_tuning.argtypes = [_int, _int, _int]
+_lib.lrd_selftest_wait_timeout.restype = _int
+_lib.lrd_selftest_wait_timeout.argtypes = [C.c_void_p]
 _lib.lrd_chain_pair_tuning.restype = _int
 _lib.lrd_chain_pair_tuning.argtypes = [_int, _int, _int, _int]
 _pp = C.POINTER(C.c_void_p)
@@ -167,6 +169,10 @@ def lrd_status_string(status):
 
 def lrd_launch_count():
     return int(_lib.lrd_launch_count())
+
+
+def lrd_selftest_wait_timeout(stream=None):
+    _check(_lib.lrd_selftest_wait_timeout(_stream(stream)))
 
 
 def lrd_set_path(path):

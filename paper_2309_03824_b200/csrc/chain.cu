@@ -427,7 +427,8 @@ int pick_bn2(int64_t N2, int C) {
 
 // Clusters of C blocks that can be resident at once (a cluster needs C free SMs inside one GPC).
 int max_active_clusters(int C) {
-    static int cache[5] = {0, 0, 0, 0, 0};
+    static int cache_on[kMaxDevices][5] = {};
+    int* cache = cache_on[device_slot()];
     if (C < 2 || C > 4) return kNumSms;
     if (cache[C] == 0) {
         int n = 0;
@@ -578,7 +579,8 @@ lrd_status_t chain_launch(const ChainArgs& a, cudaStream_t stream) {
     }
     p.timeout_flag = device_timeout_flag();
 
-    static bool configured = false;
+    static bool configured_on[kMaxDevices] = {};
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (cudaFuncSetAttribute(chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
             return LRD_ERR_CUDA;

@@ -459,7 +459,8 @@ int pick_bn2(int64_t N2, int S) {
 
 // Clusters of n blocks that can be resident at once (a cluster needs n free SMs inside one GPC).
 int max_active_clusters(int n) {
-    static int cache[2 * kMaxS + 1] = {0};
+    static int cache_on[kMaxDevices][2 * kMaxS + 1] = {};
+    int* cache = cache_on[device_slot()];
     if (n < 2 || n > 2 * kMaxS) return kNumSms;
     if (cache[n] == 0) {
         int cnt = 0;
@@ -633,7 +634,8 @@ lrd_status_t chain_pair_launch(const ChainArgs* layers, int n, cudaStream_t stre
     }
     p.timeout_flag = device_timeout_flag();
 
-    static bool configured = false;
+    static bool configured_on[kMaxDevices] = {};
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (!cuda_ok(cudaFuncSetAttribute(chain_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit), "cudaFuncSetAttribute(pair chain)"))
             return LRD_ERR_CUDA;

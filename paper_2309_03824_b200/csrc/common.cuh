@@ -8,10 +8,21 @@
 
 namespace lrd {
 
-// Device address of the flag a bounded wait raises when it runs out (one word, zero = fine);
+// Per-device host-side caches (function attributes set, occupancy answers, symbol addresses) are kept in tables
+// indexed by the current device's ordinal; devices past the table share its last row.
+constexpr int kMaxDevices = 16;
+inline int device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+    return dev < kMaxDevices ? dev : kMaxDevices - 1;
+}
+
+// Device address (on the current device) of the flag a bounded wait raises when it runs out (one word, zero = fine);
 // nullptr if the address cannot be obtained.  Read and cleared by lrd_check_device_status().
 unsigned int* device_timeout_flag();
 lrd_status_t read_and_clear_device_timeout(bool* raised);
+// One block whose bounded wait is left to run out (see lrd_selftest_wait_timeout).
+lrd_status_t selftest_wait_runs_out(cudaStream_t stream);
 
 // One matrix product  C[M x N] = op(A) op(B) (+ bias over columns), fp32 accumulate.
 //   a_mn_major = false: A stored [M x K] (k contiguous);  true: A stored [K x M] (m contiguous)

@@ -509,7 +509,8 @@ lrd_status_t tc_conv3x3(bool dgrad, const void* img, const void* G, void* out, i
     p.ka = (int)ka; p.n_total = (int)n_total; p.g_ci = (int)ci; p.sign = dgrad ? -1 : 1;
     p.out = (__nv_bfloat16*)out; p.timeout_flag = device_timeout_flag();
     p.n2 = 0; p.out2 = nullptr; p.bias2 = nullptr;
-    static bool configured = false;
+    static bool configured_on[kMaxDevices] = {};
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (!set_smem(conv_kernel<false, false>, kSmemBytes) || !set_smem(conv_kernel<true, false>, kSmemBytes)) return LRD_ERR_CUDA;
         configured = true;
@@ -547,7 +548,8 @@ lrd_status_t tc_conv3x3_chain(bool dgrad, const void* img, const void* G, const 
     p.ka = (int)ka; p.n_total = (int)n1; p.g_ci = (int)ci; p.sign = dgrad ? -1 : 1;
     p.out = (__nv_bfloat16*)core_out; p.timeout_flag = device_timeout_flag();
     p.n2 = (int)n2; p.out2 = (__nv_bfloat16*)out2; p.bias2 = (const __nv_bfloat16*)bias2;
-    static bool configured = false;
+    static bool configured_on[kMaxDevices] = {};
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (!set_smem(conv_kernel<false, true>, kSmemBytes) || !set_smem(conv_kernel<true, true>, kSmemBytes)) return LRD_ERR_CUDA;
         configured = true;
@@ -576,7 +578,8 @@ lrd_status_t tc_conv3x3_filter(const void* dout, const void* in, void* dG, int64
     p.chunks_per_split = (p.chunks_total + splits - 1) / splits;
     p.ldp = (int)((ci + 3) / 4 * 4);
     p.partial = scratch; p.timeout_flag = device_timeout_flag();
-    static bool configured = false;
+    static bool configured_on[kMaxDevices] = {};
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (!set_smem(filter_kernel, kFSmemBytes)) return LRD_ERR_CUDA;
         configured = true;

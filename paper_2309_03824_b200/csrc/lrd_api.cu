@@ -106,6 +106,37 @@ ChainArgs bwd_chain_args(const Linear& L, const void* dY, const void* V, const v
     return c;
 }
 
+// A bf16 layer whose factors are stored with leading dimensions that are not multiples of 8 elements (an unquantized
+// rank stored packed: rows start at addresses that are not multiples of 16 bytes) cannot feed TMA or the MMA
+// descriptors directly.  Its factors are small -- r (K + N) elements -- so they are copied into the workspace with
+// the rank rounded up to a multiple of 16 and zero columns, the layer runs on the tensor-core kernels at the padded
+// rank (the zero columns add nothing), and Z / dU / dV are copied between the caller's packed layout and padded
+// buffers.  The rank itself is unchanged: this is what an odd rank costs on this hardware beside a rounded one.
+bool needs_repack(const Linear& L) { return L.dt == LRD_BF16 && L.r > 0 && (L.ldv % 8 || L.ldu % 8 || L.ldz % 8); }
+int64_t padded_rank(const Linear& L) { return (L.r + 15) / 16 * 16; }
+lrd_linear_desc_t padded_desc(const lrd_linear_desc_t& d, const Linear& L) {
+    lrd_linear_desc_t q = d;
+    q.r = padded_rank(L);
+    q.ldv = q.ldu = q.ldz = q.r;
+    q.ldx = L.ldx; q.ldy = L.ldy;
+    return q;
+}
+struct RepackLayout {           // offsets into the workspace, behind the padded layer's own workspace
+    size_t inner, Vp, Up, Zp, dUp, dVp, total;
+};
+RepackLayout repack_layout(const Linear& L, size_t inner_bytes) {
+    const size_t rp = (size_t)padded_rank(L), e = 2;
+    RepackLayout o;
+    o.inner = 0;
+    o.Vp = align_up(inner_bytes, 256);
+    o.Up = o.Vp + align_up((size_t)L.K * rp * e, 256);
+    o.Zp = o.Up + align_up((size_t)L.N * rp * e, 256);
+    o.dUp = o.Zp + align_up((size_t)(L.M > 0 ? L.M : 1) * rp * e, 256);
+    o.dVp = o.dUp + align_up((size_t)L.N * rp * e, 256);
+    o.total = o.dVp + align_up((size_t)L.K * rp * e, 256);
+    return o;
+}
+
 size_t linear_z_bytes(const Linear& L) { return align_up((size_t)(L.M > 0 ? L.M : 1) * L.r * elem_size(L.dt), 256); }
 
 size_t linear_grad_scratch_bytes(const Linear& L) {     // dU, dV and dbias of one step, in the parameters' layouts
@@ -167,6 +198,30 @@ __global__ void add_into_kernel(T* __restrict__ dst, const T* __restrict__ src, 
     }
 }
 }  // namespace
+
+namespace {
+// dst[row][0 .. cols_dst) = src[row][0 .. cols_src) followed by zeros (cols_dst >= cols_src), 2-byte elements, any
+// leading dimensions: the copy between a packed factor (rows that start at odd multiples of 2 bytes) and its copy
+// with rows padded to whole 16-byte groups.
+__global__ void copy2d_bf16_kernel(__nv_bfloat16* __restrict__ dst, int64_t ldd, const __nv_bfloat16* __restrict__ src, int64_t lds,
+                                   int64_t rows, int64_t cols_src, int64_t cols_dst) {
+    const int64_t n = rows * cols_dst;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / cols_dst, c = i % cols_dst;
+        dst[r * ldd + c] = c < cols_src ? src[r * lds + c] : __float2bfloat16_rn(0.f);
+    }
+}
+}  // namespace
+
+lrd_status_t copy2d_bf16(void* dst, int64_t ldd, const void* src, int64_t lds, int64_t rows, int64_t cols_src, int64_t cols_dst,
+                         cudaStream_t s) {
+    if (rows <= 0 || cols_dst <= 0) return LRD_OK;
+    const int64_t n = rows * cols_dst;
+    const unsigned blocks = (unsigned)std::min<int64_t>((n + 255) / 256, 148 * 16);
+    copy2d_bf16_kernel<<<blocks, 256, 0, s>>>((__nv_bfloat16*)dst, ldd, (const __nv_bfloat16*)src, lds, rows, cols_src, cols_dst);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
 
 lrd_status_t add_into(void* dst, const void* src, int64_t rows, int64_t cols, int64_t ld, lrd_dtype_t dt, cudaStream_t s) {
     if (!dst || rows <= 0 || cols <= 0) return LRD_OK;
@@ -309,9 +364,18 @@ lrd_status_t lrd_check_device_status(void) {
     return raised ? LRD_ERR_TIMEOUT : LRD_OK;
 }
 
+lrd_status_t lrd_selftest_wait_timeout(void* cuda_stream) {
+    LRD_TRY(check_arch());
+    return selftest_wait_runs_out((cudaStream_t)cuda_stream);
+}
+
 size_t lrd_linear_workspace_bytes(const lrd_linear_desc_t* desc, lrd_freeze_t freeze, int is_bwd) {
     Linear L;
     if (parse_linear(desc, &L, false) != LRD_OK) return 0;
+    if (needs_repack(L)) {
+        const lrd_linear_desc_t q = padded_desc(*desc, L);
+        return repack_layout(L, lrd_linear_workspace_bytes(&q, freeze, is_bwd)).total;
+    }
     (void)freeze;
     if (!is_bwd) return linear_z_bytes(L);
     const size_t bwd = linear_z_bytes(L) + linear_split_bytes(L);
@@ -346,6 +410,18 @@ static lrd_status_t linear_fwd_on(const lrd_linear_desc_t* desc, const void* X, 
     LRD_TRY(check_ws(workspace, workspace_bytes, lrd_linear_workspace_bytes(desc, freeze, 0)));
     LRD_TRY(check_arch());
     if (L.M == 0 || check_only) return LRD_OK;
+
+    if (needs_repack(L) && g_path.load() != LRD_PATH_GENERAL && L.ldx % 8 == 0 && L.ldy % 8 == 0) {
+        const lrd_linear_desc_t q = padded_desc(*desc, L);
+        const size_t inner = lrd_linear_workspace_bytes(&q, freeze, 0);
+        const RepackLayout o = repack_layout(L, inner);
+        uint8_t* w = (uint8_t*)workspace;
+        LRD_TRY(copy2d_bf16(w + o.Vp, q.r, V, L.ldv, L.K, L.r, q.r, s));
+        LRD_TRY(copy2d_bf16(w + o.Up, q.r, U, L.ldu, L.N, L.r, q.r, s));
+        LRD_TRY(linear_fwd_on(&q, X, w + o.Vp, w + o.Up, bias, Y, Z_save ? w + o.Zp : nullptr, freeze, w, inner, s, sm_share));
+        if (Z_save) LRD_TRY(copy2d_bf16(Z_save, L.ldz, w + o.Zp, q.r, L.M, L.r, L.r, s));
+        return LRD_OK;
+    }
 
     const int path = g_path.load();
     if (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) {
@@ -397,6 +473,23 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
     if (L.M == 0) {                      // no tokens: the unfrozen gradients are sums over nothing
         if (plan & LRD_PLAN_DU) { LRD_TRY(zero_fill(dU, L.N, L.r, L.ldu, L.dt, s)); LRD_TRY(zero_fill(dbias, 1, L.N, L.N, L.dt, s)); }
         if (plan & LRD_PLAN_DV) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
+        return LRD_OK;
+    }
+
+    if (needs_repack(L) && g_path.load() != LRD_PATH_GENERAL && L.ldx % 8 == 0 && L.ldy % 8 == 0 && !data_done) {
+        const lrd_linear_desc_t q = padded_desc(*desc, L);
+        const size_t inner = lrd_linear_workspace_bytes(&q, freeze, 1);
+        const RepackLayout o = repack_layout(L, inner);
+        uint8_t* w = (uint8_t*)workspace;
+        const bool du = (plan & LRD_PLAN_DU) != 0, dv = (plan & LRD_PLAN_DV) != 0;
+        LRD_TRY(copy2d_bf16(w + o.Vp, q.r, V, L.ldv, L.K, L.r, q.r, s));
+        LRD_TRY(copy2d_bf16(w + o.Up, q.r, U, L.ldu, L.N, L.r, q.r, s));
+        if (du) LRD_TRY(copy2d_bf16(w + o.Zp, q.r, Z_save, L.ldz, L.M, L.r, q.r, s));
+        // the frozen factor's buffers were zero-filled above; the padded call gets none for them
+        LRD_TRY(linear_bwd_on(&q, dY, X, w + o.Vp, w + o.Up, du ? w + o.Zp : nullptr, dX, du ? w + o.dUp : nullptr, dv ? w + o.dVp : nullptr,
+                              du ? dbias : nullptr, freeze, w, inner, s, nullptr, nullptr, sm_share));
+        if (du) LRD_TRY(copy2d_bf16(dU, L.ldu, w + o.dUp, q.r, L.N, L.r, L.r, s));
+        if (dv) LRD_TRY(copy2d_bf16(dV, L.ldv, w + o.dVp, q.r, L.K, L.r, L.r, s));
         return LRD_OK;
     }
 
@@ -583,6 +676,8 @@ lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const v
     LRD_TRY(parse_linear(desc, &L, true));
     if (!X || !W || !Y) return LRD_ERR_INVALID_ARG;
     (void)workspace; (void)workspace_bytes;
+    for (const void* p : {X, W, bias, (const void*)Y})
+        if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
     LRD_TRY(check_arch());
     return run_gemm(gemm(L.M, L.N, L.K, X, L.ldx, false, W, L.ldv, false, Y, L.ldy, bias, L.dt), false, nullptr, 0,
                     (cudaStream_t)cuda_stream);
@@ -593,6 +688,8 @@ lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const 
     Linear L;
     LRD_TRY(parse_linear(desc, &L, true));
     if (!dY || !X || !W || !dW) return LRD_ERR_INVALID_ARG;
+    for (const void* p : {dY, X, W, (const void*)dX, (const void*)dW, (const void*)dbias})
+        if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
     LRD_TRY(check_ws(workspace, workspace_bytes, lrd_dense_workspace_bytes(desc, 1)));
     LRD_TRY(check_arch());
     cudaStream_t s = (cudaStream_t)cuda_stream;
@@ -624,6 +721,8 @@ lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, cons
     if (!X || !A || !G || !Bm || !Y) return LRD_ERR_INVALID_ARG;
     if ((freeze == LRD_TK_FREEZE_CORE) != (Z1_save == nullptr)) return LRD_ERR_INVALID_ARG;
     if ((freeze == LRD_TK_FREEZE_FACTORS) != (Z2_save == nullptr)) return LRD_ERR_INVALID_ARG;
+    for (const void* p : {X, A, G, Bm, bias, (const void*)Y, (const void*)Z1_save, (const void*)Z2_save})
+        if (p && !elem_aligned(p, desc->dtype)) return LRD_ERR_ALIGNMENT;
     LRD_TRY(check_ws(workspace, workspace_bytes, tucker2_workspace_bytes(desc, freeze, 0)));
     LRD_TRY(check_arch());
     return tucker2_fwd(desc, X, A, G, Bm, bias, Y, Z1_save, Z2_save, freeze, workspace, workspace_bytes,
@@ -638,6 +737,8 @@ lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, con
     if (!dY || !A || !G || !Bm) return LRD_ERR_INVALID_ARG;
     if (freeze != LRD_TK_FREEZE_FACTORS && (!X || !Z2_save || !dA || !dB)) return LRD_ERR_INVALID_ARG;
     if (freeze != LRD_TK_FREEZE_CORE && (!Z1_save || !dG)) return LRD_ERR_INVALID_ARG;
+    for (const void* p : {dY, X, A, G, Bm, Z1_save, Z2_save, (const void*)dX, (const void*)dA, (const void*)dG, (const void*)dB, (const void*)dbias})
+        if (p && !elem_aligned(p, desc->dtype)) return LRD_ERR_ALIGNMENT;
     LRD_TRY(check_ws(workspace, workspace_bytes, tucker2_workspace_bytes(desc, freeze, 1)));
     LRD_TRY(check_arch());
     return tucker2_bwd(desc, dY, X, A, G, Bm, Z1_save, Z2_save, dX, dA, dG, dB, dbias, freeze, workspace,

@@ -10,12 +10,14 @@ namespace lrd {
 __device__ unsigned int g_device_timeout = 0;
 
 unsigned int* device_timeout_flag() {
-    static unsigned int* ptr = nullptr;
-    if (!ptr) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_device_timeout) == cudaSuccess) ptr = (unsigned int*)p;
-    }
-    return ptr;
+    static unsigned int* ptr_on[kMaxDevices] = {};          // every device has its own copy of the symbol
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    void* p = nullptr;
+    if (dev < 0 || dev >= kMaxDevices)                      // past the table: look it up every time
+        return cudaGetSymbolAddress(&p, g_device_timeout) == cudaSuccess ? (unsigned int*)p : nullptr;
+    if (!ptr_on[dev] && cudaGetSymbolAddress(&p, g_device_timeout) == cudaSuccess) ptr_on[dev] = (unsigned int*)p;
+    return ptr_on[dev];
 }
 
 lrd_status_t read_and_clear_device_timeout(bool* raised) {
@@ -311,14 +313,14 @@ constexpr int kNoAllocMaxSplits = 64;
 constexpr size_t kNoAllocFloats = (size_t)kNoAllocMaxN * kNoAllocMaxSplits;   // 2 MiB per GPU that loads the library
 static __device__ __align__(256) float g_noalloc_scratch[kNoAllocFloats];
 
-constexpr int kMaxDevices = 64;
-float* g_noalloc_ptr[kMaxDevices] = {};                          // device address of the array, per device
+constexpr int kNoallocMaxDevices = 64;
+float* g_noalloc_ptr[kNoallocMaxDevices] = {};                          // device address of the array, per device
 
 // In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a kernel can use:
 // the device address is asked for once per device (with that device current) and cached.
 lrd_status_t noalloc_scratch(float** out) {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LRD_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoallocMaxDevices) return LRD_ERR_CUDA;
     if (!g_noalloc_ptr[dev]) {
         float* ptr = nullptr;
         if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return LRD_ERR_CUDA;

@@ -2,7 +2,6 @@
 
 namespace lrd {
 namespace {
-constexpr int kMaxDevices = 16;
 // one table per host thread: calls from different threads never share a stream or an event
 thread_local SideStreams g_sides[kMaxDevices];
 thread_local int g_n_sides = 0;

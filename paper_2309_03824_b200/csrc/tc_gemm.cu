@@ -441,7 +441,8 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
 template <int BN, bool A_MN, bool B_MN, bool ONES = false>
 lrd_status_t launch(const CUtensorMap& tA, const CUtensorMap& tB, const TcParams& p, dim3 grid, cudaStream_t stream) {
     auto kern = tc_gemm_kernel<BN, A_MN, B_MN, ONES>;
-    static bool configured = false;     // per instantiation; the attribute is sticky per function
+    static bool configured_on[kMaxDevices] = {};     // per instantiation; the attribute is sticky per function
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN, ONES>::SMEM_BYTES) != cudaSuccess)
             return LRD_ERR_CUDA;
@@ -524,7 +525,8 @@ static int global_splits(int64_t M, int64_t N, int64_t K, int bn) {
 // Clusters of S blocks that can be resident at once (S blocks need S free SMs inside one GPC, so this is
 // fewer than SMs / S).  All instantiations hold one block per SM, so one of them answers for all.
 static int max_active_clusters(int S) {
-    static int cache[kMaxClusterSplits + 1] = {0};
+    static int cache_on[kMaxDevices][kMaxClusterSplits + 1] = {};
+    int* cache = cache_on[device_slot()];
     if (S < 2 || S > kMaxClusterSplits) return kNumSms;
     if (cache[S] == 0) {
         auto kern = tc_gemm_kernel<64, true, true, false>;

@@ -282,7 +282,8 @@ template <int BN, bool A_MN, bool B_MN, int CG>
 lrd_status_t launch_p(const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tC, const PParams& p, unsigned blocks,
                       cudaStream_t stream) {
     auto kern = tc_gemm_persistent_kernel<BN, A_MN, B_MN, CG>;
-    static bool configured = false;     // per instantiation; the attribute is sticky per function
+    static bool configured_on[kMaxDevices] = {};     // per instantiation; the attribute is sticky per function
+    bool& configured = configured_on[device_slot()];
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<BN, CG>::SMEM_BYTES) != cudaSuccess)
             return LRD_ERR_CUDA;

@@ -50,6 +50,58 @@ def test_tensor_core_fused_or_auto(shape, freeze):
     check_linear(wl.random_factor_case(M, K, N, r, "bf16", 300 + M), freeze, path=b.LRD_PATH_FUSED)
 
 
+@pytest.mark.parametrize("shape", [(300, 200, 136, 5), (513, 776, 264, 33), (640, 768, 768, 100), (1100, 1032, 520, 250),
+                                   (384, 768, 3072, 390)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_packed_ranks_off_a_multiple_of_8(shape, freeze):
+    """Factors stored packed with a rank that is not a multiple of 8 (rows of V, U, Z, dU, dV start off 16-byte
+    boundaries): the factors are repacked into the workspace and the layer still runs on the tensor-core kernels."""
+    M, K, N, r = shape
+    check_linear(wl.random_factor_case(M, K, N, r, "bf16", 350 + M), freeze)
+
+
+def test_odd_factor_strides_leave_the_padding_alone():
+    M, K, N, r = 260, 136, 200, 40
+    ldv, ldu, ldz = 43, 45, 41
+    case = wl.random_factor_case(M, K, N, r, "bf16", 360)
+    code, tdt = DT["bf16"]
+    desc = b.linear_desc(M, K, N, r, code, 0, ldv, ldu, 0, ldz)
+
+    def padded(a, ld, fill=float("nan")):
+        t = torch.full((a.shape[0], ld), fill, dtype=tdt, device="cuda")
+        t[:, : a.shape[1]] = dev(a, "bf16")
+        return t
+
+    X, dY, bias = dev(case["X"], "bf16"), dev(case["dY"], "bf16"), dev(case["b"], "bf16")
+    V, U = padded(case["V"], ldv), padded(case["U"], ldu)
+    Y = torch.empty(M, N, dtype=tdt, device="cuda")
+    Z = torch.full((M, ldz), 3.0, dtype=tdt, device="cuda")
+    dX = torch.empty(M, K, dtype=tdt, device="cuda")
+    dU = torch.full((N, ldu), 3.0, dtype=tdt, device="cuda")
+    dV = torch.full((K, ldv), 3.0, dtype=tdt, device="cuda")
+    db = torch.empty(N, dtype=tdt, device="cuda")
+    ws = workspace(max(b.lrd_linear_workspace_bytes(desc, 0, 0), b.lrd_linear_workspace_bytes(desc, 0, 1)))
+    b.lrd_linear_fwd(desc, X, V, U, bias, Y, Z, b.LRD_FREEZE_NONE, ws)
+    b.lrd_linear_bwd(desc, dY, X, V, U, Z, dX, dU, dV, db, b.LRD_FREEZE_NONE, ws)
+    torch.cuda.synchronize()
+    assert b.lrd_check_device_status() == b.LRD_OK
+    ref = oracle_linear(case, b.LRD_FREEZE_NONE)
+    for got, name, w in ((Y, "Y", N), (Z, "Z", r), (dX, "dX", K), (dU, "dU", r), (dV, "dV", r), (db.reshape(1, -1), "db", N)):
+        assert rel_err(got[:, :w], np.asarray(ref[name]).reshape(got.shape[0], -1)) <= TOL["bf16"], name
+    for got, w in ((Z, r), (dU, r), (dV, r)):
+        assert (got[:, w:] == 3.0).all()                      # columns past the rank are never written
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_once():
+    """The self-test block waits on a barrier nothing arrives at; its wait gives up at the limit every pipeline wait
+    has, the status check reports LRD_ERR_TIMEOUT exactly once, and the library keeps working afterwards."""
+    assert b.lrd_check_device_status() == b.LRD_OK
+    b.lrd_selftest_wait_timeout()
+    assert b.lrd_check_device_status() == b.LRD_ERR_TIMEOUT
+    assert b.lrd_check_device_status() == b.LRD_OK
+    check_linear(wl.random_factor_case(300, 200, 136, 64, "bf16", 370), b.LRD_FREEZE_NONE)
+
+
 def _svd_factors(W, r):
     Uf, s, Vt = np.linalg.svd(W, full_matrices=False)     # input construction only
     root = np.sqrt(s[:r])

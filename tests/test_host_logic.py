@@ -77,6 +77,27 @@ def test_argument_errors_are_reported_before_any_launch():
     b.lrd_set_path(b.LRD_PATH_AUTO)
 
 
+def test_misaligned_pointers_are_rejected_before_any_launch():
+    """Every entry point checks its base pointers against the element size on the host (odd addresses for bf16,
+    addresses off a multiple of 4 for fp32) and returns LRD_ERR_ALIGNMENT without touching a device."""
+    P = ctypes.c_void_p
+    ok, odd, off2 = 0x7F0000001000, 0x7F0000001001, 0x7F0000001002
+    for dt, bad in ((b.LRD_BF16, odd), (b.LRD_F32, off2), (b.LRD_F32, odd)):
+        d = b.linear_desc(8, 16, 16, 4, dt)
+        assert b._lib.lrd_linear_fwd(ctypes.byref(d), P(ok), P(bad), P(ok), None, P(ok), P(ok), 0, P(ok), 1 << 20, None) == b.LRD_ERR_ALIGNMENT
+        assert b._lib.lrd_dense_fwd(ctypes.byref(d), P(bad), P(ok), None, P(ok), None, 0, None) == b.LRD_ERR_ALIGNMENT
+        assert b._lib.lrd_dense_fwd(ctypes.byref(d), P(ok), P(ok), P(bad), P(ok), None, 0, None) == b.LRD_ERR_ALIGNMENT
+        assert b._lib.lrd_dense_bwd(ctypes.byref(d), P(ok), P(ok), P(ok), P(ok), P(bad), None, P(ok), 1 << 20, None) == b.LRD_ERR_ALIGNMENT
+        assert b._lib.lrd_dense_bwd(ctypes.byref(d), P(ok), P(ok), P(ok), None, P(ok), P(bad), P(ok), 1 << 20, None) == b.LRD_ERR_ALIGNMENT
+        t = b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, dt)
+        assert b._lib.lrd_tucker2_fwd(ctypes.byref(t), P(ok), P(ok), P(bad), P(ok), None, P(ok), P(ok), P(ok), 0, P(ok), 1 << 20,
+                                      None) == b.LRD_ERR_ALIGNMENT
+        assert b._lib.lrd_tucker2_fwd(ctypes.byref(t), P(ok), P(ok), P(ok), P(ok), P(bad), P(ok), P(ok), P(ok), 0, P(ok), 1 << 20,
+                                      None) == b.LRD_ERR_ALIGNMENT
+        assert b._lib.lrd_tucker2_bwd(ctypes.byref(t), P(ok), P(ok), P(ok), P(ok), P(ok), P(ok), P(ok), P(ok), P(ok), P(ok), P(ok),
+                                      P(bad), 0, P(ok), 1 << 20, None) == b.LRD_ERR_ALIGNMENT
+
+
 def test_rank_search_bit_exact_against_oracle():
     """Algorithm 1 on synthetic step-time curves: the library's host routine and the oracle pick the same rank
     and take the same keep-the-original decision (staircases, ties, flat and monotone curves, one point)."""

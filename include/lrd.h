@@ -117,10 +117,39 @@ uint32_t lrd_linear_bwd_plan(lrd_freeze_t freeze);
  * r running downward, to a time not yet measured; the reading taken here: delta(r) = t(r+1) - t(r) for
  * R_min <= r < R is the time saved by stepping down to r, R_opt is the first local maximum of delta met
  * scanning down from R-1 (strictly above both neighbours and above zero; an end point has one neighbour),
- * and with no such peak the global maximum (largest r on ties).  *use_decomposed (nullable) receives 1
- * when t(R_opt) < T_orig (the algorithm's closing test: keep the original layer otherwise), else 0.
- * Returns R_opt, or -(lrd_status_t) for a null curve, n < 1 or R_min < 1.  `t` is host memory. */
-int64_t lrd_rank_search(const double* t, int64_t n, int64_t R_min, double T_orig, int* use_decomposed);
+ * and with no such peak the global maximum (largest r on ties).
+ * min_rel_drop >= 0: on a measured curve every wiggle of the timer is a local maximum of the difference, so a
+ * peak (and the fallback maximum) counts only if its drop is at least min_rel_drop * t(r); pass a multiple of the
+ * timer's relative spread (Section 2.1's example, 257 -> 256, is a drop of 15 %).  With a positive threshold and
+ * no drop that large, R_opt = R.  0 is the plain reading.
+ * *use_decomposed (nullable) receives 1 when t(R_opt) < T_orig (the algorithm's closing test: keep the
+ * original layer otherwise), else 0.  Returns R_opt, or -(lrd_status_t) for a null curve, n < 1, R_min < 1
+ * or a negative threshold.  `t` is host memory. */
+int64_t lrd_rank_search(const double* t, int64_t n, int64_t R_min, double T_orig, double min_rel_drop, int* use_decomposed);
+
+/* The quantization multiple a measured curve shows (Section 2.1, "Rank Optimization": which ranks are efficient is
+ * a property of the device): the greatest common divisor of the ranks r whose drop t(r+1) - t(r) is positive and at
+ * least min_rel_drop * t(r); 1 when there is none.  Same arguments and errors as lrd_rank_search. */
+int64_t lrd_rank_multiple(const double* t, int64_t n, int64_t R_min, double min_rel_drop);
+
+/* Starting ranks of the search, host only.  lrd_svd_rank: the largest r with r (C + S) <= C S / alpha (a C x S
+ * matrix as two factors at compression ratio alpha).  lrd_tucker_rank: Eq. 5, r1 for a [S, C, k, k] kernel at
+ * ratio alpha with r2 = beta r1 (both truncated, as the paper's [512, 512, 3, 3] -> 309 example fixes); *r2
+ * (nullable) receives r2.  lrd_tucker_rank_min: Eq. 6, the lower end of the search = Eq. 5 at alpha + 1.
+ * Negative (lrd_status_t) on non-positive arguments. */
+int64_t lrd_svd_rank(int64_t C, int64_t S, double alpha);
+int64_t lrd_tucker_rank(int64_t C, int64_t S, int64_t k, double alpha, double beta, int64_t* r2);
+int64_t lrd_tucker_rank_min(int64_t C, int64_t S, int64_t k, double alpha, double beta);
+
+/* The undecomposed 3 x 3 convolution (stride 1, zero padding 1, NHWC; kernel Wk[S][3][3][C]) that a Tucker-2 layer
+ * replaces (Eq. 4): the comparison layer of the convolutional workloads and the T of Algorithm 1's closing test.
+ * Forward Y = conv(X, Wk); backward dX (nullable: skipped) and dW.  Same conventions as the other entry points;
+ * the workspace holds the split partial sums of the filter gradient. */
+size_t lrd_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype);
+lrd_status_t lrd_conv3x3_fwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* X, const void* Wk,
+                             void* Y, void* cuda_stream);
+lrd_status_t lrd_conv3x3_bwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* dY, const void* X,
+                             const void* Wk, void* dX, void* dW, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 const char* lrd_status_string(lrd_status_t s);
 

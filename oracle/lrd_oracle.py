@@ -338,7 +338,14 @@ def tucker2_bwd(dY, X, A, G, Bm, Z1, Z2, freeze=TK_FREEZE_NONE):
 # --------------------------------------------------------------------------------------
 # Algorithm 1: rank search on a measured step-time curve   (parity unpinned)
 # --------------------------------------------------------------------------------------
-def rank_search(t, R_min, T_orig):
+def _fast_ranks(t, min_rel_drop):
+    """Indices i (rank R_min + i) that it pays to step down to: delta(r) = t(r+1) - t(r) is positive and at
+    least min_rel_drop * t(r)."""
+    delta = t[1:] - t[:-1]
+    return [i for i in range(t.shape[0] - 1) if delta[i] > 0 and delta[i] >= min_rel_drop * t[i]]
+
+
+def rank_search(t, R_min, T_orig, min_rel_drop=0.0):
     """t[i] is the step time of the layer decomposed at rank R_min + i, for R_min..R.
 
     Reading of Algorithm 1 (its printed difference refers to a time that has not been
@@ -348,6 +355,13 @@ def rank_search(t, R_min, T_orig):
     scanning down from R - 1 (a strict rise over both neighbours, an end point having
     one neighbour); with no such peak, the global argmax (largest r on ties).  The
     decomposed layer is used only if t(R_opt) < T_orig.   Returns (R_opt, use_decomposed).
+
+    min_rel_drop: on a measured curve every wiggle of the timer is a local maximum of the
+    difference; the peaks the paper means are the steps of its Fig. 2 curve (257 -> 256 is
+    15 % of the step time).  A peak therefore counts only if its drop is at least
+    min_rel_drop * t(r) -- the caller passes a multiple of the timer's measured relative
+    spread.  With a positive threshold and no drop that large anywhere, no rank is worth
+    stepping down to and R_opt = R.  min_rel_drop = 0 is the plain reading above.
     """
     t = _f64(t)
     n = t.shape[0]
@@ -355,14 +369,32 @@ def rank_search(t, R_min, T_orig):
         r_opt = R_min
         return r_opt, bool(t[0] < T_orig)
     delta = t[1:] - t[:-1]                 # delta[i] belongs to rank R_min + i
+    ok = set(_fast_ranks(t, min_rel_drop)) if min_rel_drop > 0 else None
     best = None
     for i in range(n - 2, -1, -1):
         left = delta[i - 1] if i > 0 else -np.inf
         right = delta[i + 1] if i < n - 2 else -np.inf
-        if delta[i] > left and delta[i] > right and delta[i] > 0:
+        if delta[i] > left and delta[i] > right and delta[i] > 0 and (ok is None or i in ok):
             best = i
             break
     if best is None:
-        mx = delta.max()
-        best = max(i for i in range(n - 1) if delta[i] == mx)
+        if ok is None:
+            mx = delta.max()
+            best = max(i for i in range(n - 1) if delta[i] == mx)
+        elif ok:
+            mx = max(delta[i] for i in ok)
+            best = max(i for i in ok if delta[i] == mx)
+        else:
+            best = n - 1
     return R_min + best, bool(t[best] < T_orig)
+
+
+def rank_multiple(t, R_min, min_rel_drop):
+    """The quantization multiple a measured curve shows: the greatest common divisor of the ranks it pays to step
+    down to (drops of at least min_rel_drop * t(r)); 1 when there is none.  On the paper's V100 curve the fast ranks
+    are the multiples of 8 and 16 around 256; on another device the curve says which they are."""
+    t = _f64(t)
+    g = 0
+    for i in _fast_ranks(t, min_rel_drop):
+        g = math.gcd(g, R_min + i)
+    return g if g > 0 else 1

@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_selftest_wait_timeout", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_selftest_wait_timeout", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_rank_multiple", "lrd_svd_rank", "lrd_tucker_rank", "lrd_tucker_rank_min", "lrd_conv3x3_workspace_bytes", "lrd_conv3x3_fwd", "lrd_conv3x3_bwd", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
 ]
 
 
@@ -57,7 +57,21 @@ _lib.lrd_launch_count.argtypes = []
 _lib.lrd_set_path.restype = _int
 _lib.lrd_set_path.argtypes = [_int]
 _lib.lrd_rank_search.restype = _i64
-_lib.lrd_rank_search.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double, C.POINTER(C.c_int)]
+_lib.lrd_rank_search.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double, C.c_double, C.POINTER(C.c_int)]
+_lib.lrd_rank_multiple.restype = _i64
+_lib.lrd_rank_multiple.argtypes = [C.POINTER(C.c_double), _i64, _i64, C.c_double]
+_lib.lrd_svd_rank.restype = _i64
+_lib.lrd_svd_rank.argtypes = [_i64, _i64, C.c_double]
+_lib.lrd_tucker_rank.restype = _i64
+_lib.lrd_tucker_rank.argtypes = [_i64, _i64, _i64, C.c_double, C.c_double, C.POINTER(C.c_int64)]
+_lib.lrd_tucker_rank_min.restype = _i64
+_lib.lrd_tucker_rank_min.argtypes = [_i64, _i64, _i64, C.c_double, C.c_double]
+_lib.lrd_conv3x3_workspace_bytes.restype = C.c_size_t
+_lib.lrd_conv3x3_workspace_bytes.argtypes = [_i64, _i64, _i64, _i64, _i64, _int]
+_lib.lrd_conv3x3_fwd.restype = _int
+_lib.lrd_conv3x3_fwd.argtypes = [_i64, _i64, _i64, _i64, _i64, _int] + [C.c_void_p] * 4
+_lib.lrd_conv3x3_bwd.restype = _int
+_lib.lrd_conv3x3_bwd.argtypes = [_i64, _i64, _i64, _i64, _i64, _int] + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
 _lib.lrd_chain_tuning.restype = _int
 _lib.lrd_chain_tuning.argtypes = [_int, _int, _int]
 _lib.lrd_selftest_wait_timeout.restype = _int
@@ -149,14 +163,55 @@ def lrd_tucker_freeze_for_epoch(e):
     return int(_lib.lrd_tucker_freeze_for_epoch(e))
 
 
-def lrd_rank_search(t, R_min, T_orig):
+def lrd_rank_search(t, R_min, T_orig, min_rel_drop=0.0):
     """Algorithm 1 on a measured curve: t[i] = step time at rank R_min + i.  Returns (R_opt, use_decomposed)."""
     arr = (C.c_double * len(t))(*[float(x) for x in t])
     use = C.c_int(0)
-    r = int(_lib.lrd_rank_search(arr, len(t), int(R_min), float(T_orig), C.byref(use)))
+    r = int(_lib.lrd_rank_search(arr, len(t), int(R_min), float(T_orig), float(min_rel_drop), C.byref(use)))
     if r < 0:
         raise LrdError(-r)
     return r, bool(use.value)
+
+
+def lrd_rank_multiple(t, R_min, min_rel_drop):
+    arr = (C.c_double * len(t))(*[float(x) for x in t])
+    r = int(_lib.lrd_rank_multiple(arr, len(t), int(R_min), float(min_rel_drop)))
+    if r < 0:
+        raise LrdError(-r)
+    return r
+
+
+def lrd_svd_rank(Cin, S, alpha):
+    return int(_lib.lrd_svd_rank(int(Cin), int(S), float(alpha)))
+
+
+def lrd_tucker_rank(Cin, S, k, alpha, beta=1.0):
+    r2 = C.c_int64(0)
+    r1 = int(_lib.lrd_tucker_rank(int(Cin), int(S), int(k), float(alpha), float(beta), C.byref(r2)))
+    return r1, int(r2.value)
+
+
+def lrd_tucker_rank_min(Cin, S, k, alpha, beta=1.0):
+    return int(_lib.lrd_tucker_rank_min(int(Cin), int(S), int(k), float(alpha), float(beta)))
+
+
+def lrd_conv3x3_workspace_bytes(B, H, W, Cin, S, dtype):
+    return int(_lib.lrd_conv3x3_workspace_bytes(B, H, W, Cin, S, dtype))
+
+
+def lrd_conv3x3_fwd(B, H, W, Cin, S, dtype, X, Wk, Y, stream=None, check=True):
+    st = _lib.lrd_conv3x3_fwd(B, H, W, Cin, S, dtype, _ptr(X), _ptr(Wk), _ptr(Y), _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_conv3x3_bwd(B, H, W, Cin, S, dtype, dY, X, Wk, dX, dW, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_conv3x3_bwd(B, H, W, Cin, S, dtype, _ptr(dY), _ptr(X), _ptr(Wk), _ptr(dX), _ptr(dW), w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
 
 
 def lrd_linear_bwd_plan(freeze):

@@ -466,7 +466,7 @@ bool make_plan(const ChainArgs& a, Plan* out) {
     const int kb1 = (int)((a.K1 + 63) / 64);
     Plan best{};
     bool found = false;
-    const int cands[3] = {4, 2, 1};
+    const int cands[4] = {4, 3, 2, 1};
     for (int C : cands) {
         if (g_tune_C && C != g_tune_C) continue;
         if (a.r % (16 * C)) continue;

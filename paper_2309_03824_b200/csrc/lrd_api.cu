@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 
@@ -278,30 +279,72 @@ uint32_t lrd_linear_bwd_plan(lrd_freeze_t f) {
     return plan;
 }
 
-int64_t lrd_rank_search(const double* t, int64_t n, int64_t R_min, double T_orig, int* use_decomposed) {
-    if (!t || n < 1 || R_min < 1) return -(int64_t)LRD_ERR_INVALID_ARG;
+int64_t lrd_rank_search(const double* t, int64_t n, int64_t R_min, double T_orig, double min_rel_drop, int* use_decomposed) {
+    if (!t || n < 1 || R_min < 1 || !(min_rel_drop >= 0.0)) return -(int64_t)LRD_ERR_INVALID_ARG;
+    // delta[i] = t[i + 1] - t[i] belongs to rank R_min + i, i = 0 .. n-2; with a threshold only drops of at
+    // least min_rel_drop * t[i] count
+    auto counts = [&](int64_t i) {
+        const double d = t[i + 1] - t[i];
+        return d > 0.0 && (min_rel_drop == 0.0 || d >= min_rel_drop * t[i]);
+    };
     int64_t best = -1;
     if (n == 1) {
         best = 0;
     } else {
-        // delta[i] = t[i + 1] - t[i] belongs to rank R_min + i, i = 0 .. n-2
         for (int64_t i = n - 2; i >= 0 && best < 0; --i) {
             const double d = t[i + 1] - t[i];
             const bool above_left = i == 0 || d > t[i] - t[i - 1];
             const bool above_right = i == n - 2 || d > t[i + 2] - t[i + 1];
-            if (above_left && above_right && d > 0.0) best = i;
+            if (above_left && above_right && counts(i)) best = i;
         }
-        if (best < 0) {                                   // no peak: the global maximum, largest rank on ties
+        if (best < 0 && min_rel_drop == 0.0) {            // no peak: the global maximum, largest rank on ties
             double mx = t[1] - t[0];
             best = 0;
             for (int64_t i = 1; i <= n - 2; ++i) {
                 const double d = t[i + 1] - t[i];
                 if (d >= mx) { mx = d; best = i; }
             }
+        } else if (best < 0) {                            // the largest drop among those that count; none: stay at R
+            double mx = 0.0;
+            for (int64_t i = 0; i <= n - 2; ++i) {
+                const double d = t[i + 1] - t[i];
+                if (counts(i) && (best < 0 || d >= mx)) { mx = d; best = i; }
+            }
+            if (best < 0) best = n - 1;
         }
     }
     if (use_decomposed) *use_decomposed = t[best] < T_orig ? 1 : 0;
     return R_min + best;
+}
+
+int64_t lrd_rank_multiple(const double* t, int64_t n, int64_t R_min, double min_rel_drop) {
+    if (!t || n < 1 || R_min < 1 || !(min_rel_drop >= 0.0)) return -(int64_t)LRD_ERR_INVALID_ARG;
+    int64_t g = 0;
+    for (int64_t i = 0; i + 1 < n; ++i) {
+        const double d = t[i + 1] - t[i];
+        if (!(d > 0.0 && d >= min_rel_drop * t[i])) continue;
+        int64_t a = g, b = R_min + i;                     // gcd
+        while (b) { const int64_t r = a % b; a = b; b = r; }
+        g = a;
+    }
+    return g > 0 ? g : 1;
+}
+
+int64_t lrd_svd_rank(int64_t C, int64_t S, double alpha) {
+    if (C < 1 || S < 1 || !(alpha > 0.0)) return -(int64_t)LRD_ERR_INVALID_ARG;
+    return (int64_t)floor((double)C * (double)S / (alpha * (double)(C + S)));
+}
+
+int64_t lrd_tucker_rank(int64_t C, int64_t S, int64_t k, double alpha, double beta, int64_t* r2) {
+    if (C < 1 || S < 1 || k < 1 || !(alpha > 0.0) || !(beta > 0.0)) return -(int64_t)LRD_ERR_INVALID_ARG;
+    const double q = ((double)C + beta * (double)S) / (beta * (double)k * (double)k);
+    const int64_t r1 = (int64_t)floor(0.5 * (-q + sqrt(q * q + 4.0 * (double)C * (double)S / (beta * alpha))));
+    if (r2) *r2 = (int64_t)floor(beta * (double)r1);
+    return r1;
+}
+
+int64_t lrd_tucker_rank_min(int64_t C, int64_t S, int64_t k, double alpha, double beta) {
+    return lrd_tucker_rank(C, S, k, alpha + 1.0, beta, nullptr);
 }
 
 const char* lrd_status_string(lrd_status_t s) {
@@ -329,7 +372,7 @@ lrd_status_t lrd_set_path(lrd_path_t path) {
 }
 
 lrd_status_t lrd_chain_tuning(int cluster_blocks, int kblocks_per_stage, int chunk_columns) {
-    if (cluster_blocks != 0 && cluster_blocks != 1 && cluster_blocks != 2 && cluster_blocks != 4) return LRD_ERR_INVALID_ARG;
+    if (cluster_blocks < 0 || cluster_blocks > 4) return LRD_ERR_INVALID_ARG;
     if (kblocks_per_stage < 0 || kblocks_per_stage > 4) return LRD_ERR_INVALID_ARG;
     if (chunk_columns != 0 && chunk_columns != 64 && chunk_columns != 128 && chunk_columns != 192 && chunk_columns != 256) return LRD_ERR_INVALID_ARG;
     chain_tuning(cluster_blocks, kblocks_per_stage, chunk_columns);
@@ -708,6 +751,44 @@ lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const 
     LRD_TRY(run_gemm(gw, true, partials, workspace_bytes - 256, s));
     if (dbias && !db_done) LRD_TRY(colsum(dY, L.ldy, L.M, L.N, dbias, L.dt, partials, workspace_bytes - 256, s));
     return LRD_OK;
+}
+
+// ---- the undecomposed 3x3 convolution (the layer a Tucker-2 layer replaces) ---------------------------------------
+static lrd_status_t conv3x3_check(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype) {
+    if (B < 0 || H < 1 || W < 1 || C < 1 || S < 1) return LRD_ERR_INVALID_ARG;
+    if (dtype != LRD_F32 && dtype != LRD_BF16) return LRD_ERR_INVALID_ARG;
+    if (H > 32767 || W > 32767) return LRD_ERR_UNSUPPORTED;
+    return LRD_OK;
+}
+
+size_t lrd_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype) {
+    if (conv3x3_check(B, H, W, C, S, dtype) != LRD_OK) return 0;
+    return align_up(dtype == LRD_BF16 ? tc_conv_filter_scratch_bytes(B, H, W, C, S) : 0, 256) + 256;
+}
+
+lrd_status_t lrd_conv3x3_fwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* X, const void* Wk,
+                             void* Y, void* cuda_stream) {
+    LRD_TRY(conv3x3_check(B, H, W, C, S, dtype));
+    if (!X || !Wk || !Y) return LRD_ERR_INVALID_ARG;
+    for (const void* p : {X, Wk, (const void*)Y})
+        if (!elem_aligned(p, dtype)) return LRD_ERR_ALIGNMENT;
+    LRD_TRY(check_arch());
+    if (B == 0) return LRD_OK;
+    return conv3x3_fwd(X, Wk, Y, B, H, W, C, S, (lrd_dtype_t)dtype, g_path.load(), (cudaStream_t)cuda_stream);
+}
+
+lrd_status_t lrd_conv3x3_bwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* dY, const void* X,
+                             const void* Wk, void* dX, void* dW, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    LRD_TRY(conv3x3_check(B, H, W, C, S, dtype));
+    if (!dY || !X || !Wk || !dW) return LRD_ERR_INVALID_ARG;
+    for (const void* p : {dY, X, Wk, (const void*)dX, (const void*)dW})
+        if (p && !elem_aligned(p, dtype)) return LRD_ERR_ALIGNMENT;
+    LRD_TRY(check_ws(workspace, workspace_bytes, lrd_conv3x3_workspace_bytes(B, H, W, C, S, dtype)));
+    LRD_TRY(check_arch());
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (B == 0) return zero_fill(dW, S, 9 * C, 9 * C, (lrd_dtype_t)dtype, s);
+    if (dX) LRD_TRY(conv3x3_bwd_data(dY, Wk, dX, B, H, W, C, S, (lrd_dtype_t)dtype, g_path.load(), s));
+    return conv3x3_bwd_filter(dY, X, dW, B, H, W, C, S, (lrd_dtype_t)dtype, g_path.load(), (float*)workspace, workspace_bytes - 256, s);
 }
 
 size_t lrd_tucker2_workspace_bytes(const lrd_tucker2_desc_t* desc, lrd_tucker_freeze_t freeze, int is_bwd) {

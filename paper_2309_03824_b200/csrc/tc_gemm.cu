@@ -11,9 +11,11 @@
 //                     (tiles wider than the cluster path supports, or more splits than a cluster holds).
 //   No floating-point atomics anywhere: weight gradients are bit-reproducible.
 //
-// One 128 x BN output tile per block.  Warp 0 issues TMA loads, warp 1 owns tensor memory and
-// issues the MMAs, warps 2-5 read the accumulator (each its own quarter of the 128 lanes) and
-// store.  The single-thread instructions are issued under elect.sync by a converged warp.  Both
+// One 128 x BN output tile per block.  Warp 0 issues the TMA loads of the A operand and warp 6 those of the
+// B operand (issuing a copy costs a thread about a hundred clocks, and an MN-major operand takes one copy per
+// 64 columns: one warp alone issues a 40 KB stage in about 0.4 us, less than the memory system delivers),
+// warp 1 owns tensor memory and issues the MMAs, warps 2-5 read the accumulator (each its own quarter of the
+// 128 lanes) and store.  The single-thread instructions are issued under elect.sync by a converged warp.  Both
 // operands may be K-major (reduction index contiguous) or MN-major (row / column index contiguous),
 // which covers every product of the forward and backward pass without a transposed copy.
 #include <algorithm>
@@ -29,7 +31,7 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;                         // warp 6: second TMA producer (the B operand)
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
 constexpr int kMaxClusterSplits = 8;                 // portable cluster size
 
@@ -129,13 +131,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t b_dst = a_dst + A_STAGE_BYTES;
             const int k0 = kb * BK;
             if (elect_one()) {
-                mbar_expect_tx(fb, A_STAGE_BYTES + BN * BK * 2);
+                mbar_expect_tx(fb, A_STAGE_BYTES + BN * BK * 2);       // the whole stage: warp 6's copies complete on the same barrier
                 if (A_MN) {
 #pragma unroll
                     for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * 8192, &tmA, fb, m0 + 64 * j, k0);
                 } else {
                     tma_load_2d(a_dst, &tmA, fb, k0, m0);
                 }
+            }
+            __syncwarp();
+            (void)b_dst;
+        }
+        if (p.cluster_splits > 1) { cluster_arrive(); cluster_wait(); cluster_arrive_relaxed(); }   // barriers 1 and 2, see the epilogue
+    } else if (warp == 6) {
+        // second TMA producer: the B operand of every stage (its bytes are counted by warp 0's expect_tx; a copy that
+        // lands before that arrival only makes the barrier's byte count negative for a moment)
+        int it = 0;
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1;
+            if (!mbar_wait_uniform(smem_u32(&empty_bar[s]), ph ^ 1, ab)) break;
+            const uint32_t fb = smem_u32(&full_bar[s]);
+            const uint32_t b_dst = smem_base + s * C::STAGE_BYTES + A_STAGE_BYTES;
+            const int k0 = kb * BK;
+            if (elect_one()) {
                 if (B_MN) {
 #pragma unroll
                     for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, fb, n0 + 64 * j, k0);
@@ -145,7 +164,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             __syncwarp();
         }
-        if (p.cluster_splits > 1) { cluster_arrive(); cluster_wait(); cluster_arrive_relaxed(); }   // barriers 1 and 2, see the epilogue
+        if (p.cluster_splits > 1) { cluster_arrive(); cluster_wait(); cluster_arrive_relaxed(); }
     } else if (warp == 1) {
         // MMA issuer: converged warp, elect.sync around the issue
         const uint32_t idesc = idesc_bf16(BN + ((ONES && blockIdx.x == 0) ? 16 : 0), A_MN, B_MN);

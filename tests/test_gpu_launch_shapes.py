@@ -19,6 +19,7 @@ pytestmark = pytest.mark.gpu
 def _restore_tuning():
     yield
     b.lrd_chain_tuning(0, 0, 0)
+    b.lrd_chain_pair_tuning(0, 0, 0, 0)
     b.lrd_gemm_tuning(0)
     b.lrd_set_path(b.LRD_PATH_AUTO)
 
@@ -35,8 +36,36 @@ def test_chain_kernel_launch_shape_overrides(tune, shape):
     assert b.lrd_launch_count() - n0 == 4          # fused forward, fused dZ -> dX, dU (+ db), dV: the override stayed feasible
 
 
+@pytest.mark.parametrize("shape", [(400, 776, 520, 192), (640, 768, 768, 96), (300, 776, 1000, 384)])
+def test_chain_kernel_clusters_of_three(shape):
+    M, K, N, r = shape
+    b.lrd_chain_tuning(3, 0, 0)
+    b.lrd_chain_pair_tuning(1, 0, 0, 0)
+    try:
+        n0 = b.lrd_launch_count()
+        check_linear(wl.random_factor_case(M, K, N, r, "bf16", 930 + M), b.LRD_FREEZE_NONE, path=b.LRD_PATH_FUSED)
+        assert b.lrd_launch_count() - n0 == 4
+    finally:
+        b.lrd_chain_pair_tuning(0, 0, 0, 0)
+
+
+@pytest.mark.parametrize("mode", [(2, 1, 0, 0), (2, 2, 0, 0), (2, 3, 0, 0), (2, 4, 0, 0), (2, 0, 1, 0), (2, 0, 2, 0), (2, 2, 1, 128), (2, 1, 3, 64),
+                                  (2, 0, 0, 192)])
+@pytest.mark.parametrize("shape", [(400, 776, 520, 192), (300, 520, 1000, 384), (1100, 3072, 136, 128)])
+def test_chain_on_pairs_of_sms_launch_shape_overrides(mode, shape):
+    """The chain on pairs of SMs under forced pairs per cluster, k-blocks per stage and chunk widths (a shape an override
+    makes infeasible runs the unfused products instead: parity must hold either way)."""
+    M, K, N, r = shape
+    b.lrd_chain_pair_tuning(*mode)
+    try:
+        for freeze in (b.LRD_FREEZE_NONE, b.LRD_FREEZE_U):
+            check_linear(wl.random_factor_case(M, K, N, r, "bf16", 940 + M + mode[1]), freeze)
+    finally:
+        b.lrd_chain_pair_tuning(0, 0, 0, 0)
+
+
 def test_chain_tuning_rejects_values_outside_the_lists():
-    for bad in ((3, 0, 0), (5, 0, 0), (-1, 0, 0), (0, 5, 0), (0, -1, 0), (0, 0, 100), (0, 0, 512)):
+    for bad in ((5, 0, 0), (-1, 0, 0), (0, 5, 0), (0, -1, 0), (0, 0, 100), (0, 0, 512)):
         with pytest.raises(b.LrdError):
             b.lrd_chain_tuning(*bad)
     b.lrd_chain_tuning(0, 0, 0)

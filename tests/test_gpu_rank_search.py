@@ -14,11 +14,13 @@ def test_rank_search_on_measured_curve_matches_oracle():
     M, K, N = 512, 256, 320
     R, R_min = rs.fc_rank(K, N, 2), rs.fc_rank(K, N, 3)
     assert (R, R_min) == (71, 47) and R == o.svd_rank(K, N, 2) and R_min == o.svd_rank(K, N, 3)
-    r_opt, use, curve, T = rs.search(M, K, N, R, R_min, iters=4)
+    r_opt, use, curve, T, floor, mult = rs.search(M, K, N, R, R_min, iters=4)
     assert sorted(curve) == list(range(R_min, R + 1)) and all(v > 0 for v in curve.values()) and T > 0
-    want = o.rank_search([curve[r] for r in range(R_min, R + 1)], R_min, T)
-    assert (r_opt, use) == want
-    assert R_min <= r_opt < R or R == R_min
+    t = [curve[r] for r in range(R_min, R + 1)]
+    assert floor >= rs.MIN_DROP
+    assert (r_opt, use) == o.rank_search(t, R_min, T, floor)
+    assert mult == o.rank_multiple(t, R_min, floor)
+    assert R_min <= r_opt <= R
     assert b.lrd_check_device_status() == b.LRD_OK
 
 
@@ -26,8 +28,9 @@ def test_tucker_rank_search_on_measured_curve_matches_oracle():
     B, H, C, S = 2, 6, 48, 64
     R, R_min = rs.tucker_rank(C, S, 3, 2), rs.tucker_rank(C, S, 3, 3)
     assert (R, R_min) == (o.tucker_rank(C, S, 3, 2)[0], o.tucker_rank_min(C, S, 3, 2)) and R_min < R
-    r_opt, curve = rs.search_tucker(B, H, H, C, S, R, R_min, iters=3)
-    assert sorted(curve) == list(range(R_min, R + 1)) and all(v > 0 for v in curve.values())
-    want, _ = o.rank_search([curve[r] for r in range(R_min, R + 1)], R_min, float("inf"))
-    assert r_opt == want and R_min <= r_opt <= R
+    r_opt, use, curve, T, floor, mult = rs.search_tucker(B, H, H, C, S, R, R_min, iters=3)
+    assert sorted(curve) == list(range(R_min, R + 1)) and all(v > 0 for v in curve.values()) and T > 0
+    t = [curve[r] for r in range(R_min, R + 1)]
+    assert (r_opt, use) == o.rank_search(t, R_min, T, floor) and R_min <= r_opt <= R
+    assert mult == o.rank_multiple(t, R_min, floor)
     assert b.lrd_check_device_status() == b.LRD_OK

@@ -111,6 +111,30 @@ def test_c3_resnet_stage3_shape_full_size(freeze):
     check_tucker(case, freeze)
 
 
+@pytest.mark.parametrize("dtype,geom", [("bf16", (2, 7, 7, 64, 72)), ("bf16", (3, 14, 14, 256, 256)), ("bf16", (1, 7, 7, 512, 512)),
+                                        ("f32", (2, 5, 7, 12, 10))])
+def test_undecomposed_3x3_convolution(dtype, geom):
+    """The comparison layer (the convolution a Tucker-2 layer replaces): forward, input gradient and filter gradient
+    against the oracle's direct convolution."""
+    B, H, W, C, S = geom
+    code, tdt = DT[dtype]
+    X = wl.round_to(wl.normal(801, (B, H, W, C)), dtype)
+    Wk = wl.round_to(wl.normal(802, (S, 3, 3, C), (9 * C) ** -0.5), dtype)
+    dY = wl.round_to(wl.normal(803, (B, H, W, S)), dtype)
+    Xd, Wd, dYd = dev(X, dtype), dev(Wk, dtype), dev(dY, dtype)
+    Y = torch.full((B, H, W, S), float("nan"), dtype=tdt, device="cuda")
+    dX = torch.full((B, H, W, C), float("nan"), dtype=tdt, device="cuda")
+    dW = torch.full((S, 3, 3, C), float("nan"), dtype=tdt, device="cuda")
+    ws = workspace(b.lrd_conv3x3_workspace_bytes(B, H, W, C, S, code))
+    b.lrd_conv3x3_fwd(B, H, W, C, S, code, Xd, Wd, Y)
+    b.lrd_conv3x3_bwd(B, H, W, C, S, code, dYd, Xd, Wd, dX, dW, ws)
+    torch.cuda.synchronize()
+    assert b.lrd_check_device_status() == b.LRD_OK
+    assert rel_err(Y, o.conv2d_nhwc_fwd(X, Wk, 1)) <= TOL[dtype]
+    assert rel_err(dX, o.conv2d_nhwc_bwd_data(dY, Wk, 1, (H, W))) <= TOL[dtype]
+    assert rel_err(dW, o.conv2d_nhwc_bwd_filter(dY, X, 3, 1)) <= TOL[dtype]
+
+
 def test_argument_checks():
     code, tdt = DT["bf16"]
     d = b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, code)

@@ -117,13 +117,40 @@ def test_rank_search_bit_exact_against_oracle():
             curves.append(rng.random(n))
     for t in curves:
         for T in (0.5, float(np.median(t)), 10.0):
-            want = o.rank_search(t, 100, T)
-            got = b.lrd_rank_search(t, 100, T)
-            assert got == want, (t, T, got, want)
+            for floor in (0.0, 0.02, 0.1, 0.5):
+                want = o.rank_search(t, 100, T, floor)
+                got = b.lrd_rank_search(t, 100, T, floor)
+                assert got == want, (t, T, floor, got, want)
+        for floor in (0.0, 0.02, 0.1):
+            assert b.lrd_rank_multiple(t, 100, floor) == o.rank_multiple(t, 100, floor)
     with pytest.raises(b.LrdError):
         b.lrd_rank_search([], 100, 1.0)
     with pytest.raises(b.LrdError):
         b.lrd_rank_search([1.0, 2.0], 0, 1.0)
+    with pytest.raises(b.LrdError):
+        b.lrd_rank_search([1.0, 2.0], 100, 1.0, -0.5)
+
+
+def test_rank_search_with_a_noise_floor_picks_the_cliff_not_the_first_wiggle():
+    """A staircase with the paper's 15 % step at 256 and at 248 under 1 % timer noise: the plain reading stops at the
+    first wiggle below the starting rank, the reading with a noise floor picks 256, the multiple comes out as 8, and a
+    flat noisy curve keeps the starting rank."""
+    import numpy as np
+    rng = np.random.default_rng(5)
+    R_min, R = 240, 263
+    ranks = np.arange(R_min, R + 1)
+    clean = np.where(ranks <= 248, 0.85, np.where(ranks <= 256, 1.0, 1.15))
+    hits = 0
+    for trial in range(50):
+        t = clean * (1.0 + 0.01 * rng.standard_normal(ranks.shape[0]))
+        for fn in (lambda *a: o.rank_search(*a), lambda *a: b.lrd_rank_search(*a)):
+            assert fn(t, R_min, 2.0, 0.05) == (256, True)
+        hits += o.rank_search(t, R_min, 2.0)[0] == 256
+        assert o.rank_multiple(t, R_min, 0.05) == 8 == b.lrd_rank_multiple(t, R_min, 0.05)
+        flat = 1.0 + 0.01 * rng.standard_normal(ranks.shape[0])
+        assert o.rank_search(flat, R_min, 2.0, 0.05)[0] == R == b.lrd_rank_search(flat, R_min, 2.0, 0.05)[0]
+        assert o.rank_multiple(flat, R_min, 0.05) == 1
+    assert hits < 25          # the plain reading mostly stops at timer noise: this is what the floor is for
 
 
 def test_rank_formulas_of_the_search_driver_match_the_oracle():
@@ -131,8 +158,15 @@ def test_rank_formulas_of_the_search_driver_match_the_oracle():
     paper's worked example."""
     from paper_2309_03824_b200 import rank_search as rs        # imports torch, makes no CUDA call at import
     assert rs.tucker_rank(512, 512, 3, 2) == 309 and rs.tucker_rank(512, 512, 3, 3) == o.tucker_rank_min(512, 512, 3, 2)
+    assert b.lrd_tucker_rank(512, 512, 3, 2) == (309, 309) and b.lrd_tucker_rank_min(512, 512, 3, 2) == 244
     for C in (16, 64, 96, 256, 512, 2048):
         for S in (16, 48, 256, 512, 1024):
-            for alpha in (2, 3, 4, 8):
+            for alpha in (2, 3, 4, 8, 2.5):
+                for k in (1, 3, 5):
+                    for beta in (1.0, 0.5, 2.0):
+                        assert b.lrd_tucker_rank(C, S, k, alpha, beta) == o.tucker_rank(C, S, k, alpha, beta), (C, S, k, alpha, beta)
+                        assert b.lrd_tucker_rank_min(C, S, k, alpha, beta) == o.tucker_rank_min(C, S, k, alpha, beta)
+                assert b.lrd_svd_rank(C, S, alpha) == o.svd_rank(C, S, alpha)
                 assert rs.tucker_rank(C, S, 3, alpha) == max(o.tucker_rank(C, S, 3, alpha)[0], 1), (C, S, alpha)
                 assert rs.fc_rank(C, S, alpha) == max(o.svd_rank(C, S, alpha), 1), (C, S, alpha)
+    assert b.lrd_svd_rank(0, 4, 2) < 0 and b.lrd_tucker_rank(4, 4, 3, 0.0)[0] < 0

@@ -66,5 +66,8 @@ lrd_status_t run_gemm(const GemmArgs& g, int path, bool allow_split, float* part
 GemmArgs make_gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
                    bool b_mn, void* C, int64_t ldc, const void* bias, lrd_dtype_t dt);
 lrd_status_t zero_fill(void* p, int64_t rows, int64_t cols, int64_t ld, lrd_dtype_t dt, cudaStream_t s);
+// dst[row][0 .. cols_dst) = src[row][0 .. min(cols_src, cols_dst)) then zeros; bf16, any leading dimensions.
+lrd_status_t copy2d_bf16(void* dst, int64_t ldd, const void* src, int64_t lds, int64_t rows, int64_t cols_src, int64_t cols_dst,
+                         cudaStream_t s);
 
 }  // namespace lrd

@@ -47,6 +47,30 @@ size_t split_bytes(const Tk& t) {
 
 bool g_tucker_overlap = true;
 
+// Ranks that are not multiples of 8 (rows of A, Bm, G, Z1, Z2 then start off 16-byte boundaries): as for the linear
+// layer, the factors -- small -- are copied into the workspace with the ranks rounded up to multiples of 16 and
+// zeros in the padding, the layer runs on the tensor-core kernels at the padded ranks, and Z1 / Z2 / dA / dG / dB
+// are copied between the caller's packed layout and padded buffers.
+bool needs_repack(const Tk& t) { return t.dt == LRD_BF16 && (t.r1 % 8 || t.r2 % 8) && t.C % 8 == 0 && t.S % 8 == 0; }
+int64_t pad16(int64_t r) { return (r + 15) / 16 * 16; }
+lrd_tucker2_desc_t padded_desc(const lrd_tucker2_desc_t& d) {
+    lrd_tucker2_desc_t q = d;
+    q.r1 = pad16(d.r1); q.r2 = pad16(d.r2);
+    return q;
+}
+struct Repack { size_t A, G, Bm, Z1, Z2, dA, dG, dB, total; };
+Repack repack_layout(const Tk& t, size_t inner) {
+    const size_t r1 = (size_t)pad16(t.r1), r2 = (size_t)pad16(t.r2), P = (size_t)(t.P > 0 ? t.P : 1), e = 2;
+    Repack o;
+    size_t at = align_up(inner, 256);
+    auto take = [&at](size_t bytes) { const size_t here = at; at += align_up(bytes, 256); return here; };
+    o.A = take((size_t)t.C * r1 * e); o.G = take(r2 * 9 * r1 * e); o.Bm = take((size_t)t.S * r2 * e);
+    o.Z1 = take(P * r1 * e); o.Z2 = take(P * r2 * e);
+    o.dA = take((size_t)t.C * r1 * e); o.dG = take(r2 * 9 * r1 * e); o.dB = take((size_t)t.S * r2 * e);
+    o.total = at;
+    return o;
+}
+
 #define LRD_TRY(expr)                          \
     do {                                       \
         lrd_status_t st__ = (expr);            \
@@ -70,15 +94,34 @@ lrd_status_t tucker2_check(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t free
 size_t tucker2_workspace_bytes(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t freeze, int is_bwd) {
     if (tucker2_check(d, freeze) != LRD_OK) return 0;
     const Tk t = parse(d);
+    if (needs_repack(t)) {
+        const lrd_tucker2_desc_t q = padded_desc(*d);
+        return repack_layout(t, tucker2_workspace_bytes(&q, freeze, is_bwd)).total;
+    }
     return act_bytes(t, t.r1) + act_bytes(t, t.r2) + (is_bwd ? split_bytes(t) : 0);
 }
 
 lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void* A, const void* G, const void* Bm,
                          const void* bias, void* Y, void* Z1_save, void* Z2_save, lrd_tucker_freeze_t freeze,
                          void* ws, size_t ws_bytes, int path, cudaStream_t s) {
-    (void)freeze; (void)ws_bytes;
+    (void)ws_bytes;
     const Tk t = parse(d);
     if (t.P == 0) return LRD_OK;
+    if (needs_repack(t) && path != LRD_PATH_GENERAL) {
+        const lrd_tucker2_desc_t q = padded_desc(*d);
+        const size_t inner = tucker2_workspace_bytes(&q, freeze, 0);
+        const Repack o = repack_layout(t, inner);
+        uint8_t* w = (uint8_t*)ws;
+        LRD_TRY(copy2d_bf16(w + o.A, q.r1, A, t.r1, t.C, t.r1, q.r1, s));
+        LRD_TRY(copy2d_bf16(w + o.G, q.r1, G, t.r1, t.r2 * 9, t.r1, q.r1, s));
+        LRD_TRY(zero_fill(w + o.G + (size_t)t.r2 * 9 * q.r1 * 2, (q.r2 - t.r2) * 9, q.r1, q.r1, LRD_BF16, s));
+        LRD_TRY(copy2d_bf16(w + o.Bm, q.r2, Bm, t.r2, t.S, t.r2, q.r2, s));
+        LRD_TRY(tucker2_fwd(&q, X, w + o.A, w + o.G, w + o.Bm, bias, Y, Z1_save ? w + o.Z1 : nullptr, Z2_save ? w + o.Z2 : nullptr, freeze,
+                            w, inner, path, s));
+        if (Z1_save) LRD_TRY(copy2d_bf16(Z1_save, t.r1, w + o.Z1, q.r1, t.P, q.r1, t.r1, s));
+        if (Z2_save) LRD_TRY(copy2d_bf16(Z2_save, t.r2, w + o.Z2, q.r2, t.P, q.r2, t.r2, s));
+        return LRD_OK;
+    }
     void* Z1 = Z1_save ? Z1_save : ws;
     void* Z2 = Z2_save ? Z2_save : (void*)((uint8_t*)ws + act_bytes(t, t.r1));
     LRD_TRY(run_gemm(make_gemm(t.P, t.r1, t.C, X, t.C, false, A, t.r1, true, Z1, t.r1, nullptr, t.dt), path, false, nullptr, 0, s));
@@ -105,6 +148,28 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
     }
     if (!core || t.P == 0) LRD_TRY(zero_fill(dG, t.r2, 9 * t.r1, 9 * t.r1, t.dt, s));
     if (t.P == 0) return LRD_OK;
+    if (needs_repack(t) && path != LRD_PATH_GENERAL) {
+        const lrd_tucker2_desc_t q = padded_desc(*d);
+        const size_t inner = tucker2_workspace_bytes(&q, freeze, 1);
+        const Repack o = repack_layout(t, inner);
+        uint8_t* w = (uint8_t*)ws;
+        LRD_TRY(copy2d_bf16(w + o.A, q.r1, A, t.r1, t.C, t.r1, q.r1, s));
+        LRD_TRY(copy2d_bf16(w + o.G, q.r1, G, t.r1, t.r2 * 9, t.r1, q.r1, s));
+        LRD_TRY(zero_fill(w + o.G + (size_t)t.r2 * 9 * q.r1 * 2, (q.r2 - t.r2) * 9, q.r1, q.r1, LRD_BF16, s));
+        LRD_TRY(copy2d_bf16(w + o.Bm, q.r2, Bm, t.r2, t.S, t.r2, q.r2, s));
+        if (core) LRD_TRY(copy2d_bf16(w + o.Z1, q.r1, Z1_save, t.r1, t.P, t.r1, q.r1, s));
+        if (factors) LRD_TRY(copy2d_bf16(w + o.Z2, q.r2, Z2_save, t.r2, t.P, t.r2, q.r2, s));
+        // the frozen group's buffers were zero-filled above; the padded call gets none for them
+        LRD_TRY(tucker2_bwd(&q, dY, X, w + o.A, w + o.G, w + o.Bm, core ? w + o.Z1 : nullptr, factors ? w + o.Z2 : nullptr, dX,
+                            factors ? w + o.dA : nullptr, core ? w + o.dG : nullptr, factors ? w + o.dB : nullptr, factors ? dbias : nullptr,
+                            freeze, w, inner, path, s));
+        if (factors) {
+            LRD_TRY(copy2d_bf16(dA, t.r1, w + o.dA, q.r1, t.C, q.r1, t.r1, s));
+            LRD_TRY(copy2d_bf16(dB, t.r2, w + o.dB, q.r2, t.S, q.r2, t.r2, s));
+        }
+        if (core) LRD_TRY(copy2d_bf16(dG, t.r1, w + o.dG, q.r1, t.r2 * 9, q.r1, t.r1, s));
+        return LRD_OK;
+    }
 
     void* dZ1 = ws;
     void* dZ2 = (uint8_t*)ws + act_bytes(t, t.r1);

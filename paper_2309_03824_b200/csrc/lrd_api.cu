@@ -201,7 +201,7 @@ __global__ void add_into_kernel(T* __restrict__ dst, const T* __restrict__ src, 
 }  // namespace
 
 namespace {
-// dst[row][0 .. cols_dst) = src[row][0 .. cols_src) followed by zeros (cols_dst >= cols_src), 2-byte elements, any
+// dst[row][0 .. cols_dst) = src[row][0 .. min(cols_src, cols_dst)) followed by zeros, 2-byte elements, any
 // leading dimensions: the copy between a packed factor (rows that start at odd multiples of 2 bytes) and its copy
 // with rows padded to whole 16-byte groups.
 __global__ void copy2d_bf16_kernel(__nv_bfloat16* __restrict__ dst, int64_t ldd, const __nv_bfloat16* __restrict__ src, int64_t lds,

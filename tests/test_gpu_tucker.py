@@ -83,6 +83,14 @@ def test_tensor_core_path_ranks_above_128(geom, freeze):
     check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 700 + r1), freeze)
 
 
+@pytest.mark.parametrize("geom", [(2, 7, 7, 512, 512, 309, 309), (3, 14, 14, 64, 72, 33, 41), (2, 9, 11, 128, 136, 100, 96)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_ranks_off_a_multiple_of_8_run_on_the_tensor_cores(geom, freeze):
+    """Packed factors with odd ranks (Eq. 5's own 309 among them): repacked into the workspace with padded ranks."""
+    B, H, W, C, S, r1, r2 = geom
+    check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 750 + r1), freeze)
+
+
 @pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 5, 7, 12, 10, 5, 6)])
 @pytest.mark.parametrize("freeze", MASKS)
 def test_backward_launches_side_by_side_or_in_a_row_give_the_same_bits(geom, freeze):

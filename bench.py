@@ -734,6 +734,9 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "general", "unfused", "fused"])
     ap.add_argument("--groups", default="qkv", choices=["none", "qkv"],
                     help="qkv: the three independent attention projections go out as one group (the default); none: one call per layer")
+    ap.add_argument("--wgrad", default="beside", choices=["beside", "inline"],
+                    help="beside: a layer's weight gradients run on a second stream beside the next layer's data pass (lrd_linear_bwd_data + "
+                         "lrd_linear_bwd_weights; the step ends when both streams have finished); inline: one lrd_linear_bwd call per layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every step instead of CUDA graphs")
     ap.add_argument("--single-step-graphs", action="store_true", help="one CUDA graph per step instead of one per cycle of steps (every buffer set under both masks)")
@@ -822,15 +825,37 @@ def main():
                                [st["dX"] for st in sts], None if fu else [L["dU"] for L in Ls], None if fv else [L["dV"] for L in Ls],
                                None if fu else [L["db"] for L in Ls], freeze, [L["ws"] for L in Ls])
 
+    def bwd_data(L, st, freeze):
+        b.lrd_linear_bwd_data(L["desc"], st["dY"], L["V"], L["U"], st["dX"], freeze, L["ws"])
+
+    def bwd_weights(L, st, freeze):
+        b.lrd_linear_bwd_weights(L["desc"], st["dY"], None if freeze == b.LRD_FREEZE_V else st["X"], None if freeze == b.LRD_FREEZE_U else st["Z"],
+                                 None if freeze == b.LRD_FREEZE_U else L["dU"], None if freeze == b.LRD_FREEZE_V else L["dV"],
+                                 None if freeze == b.LRD_FREEZE_U else L["db"], freeze, L["ws"])
+
+    # Nothing later in the backward pass waits for a layer's weight gradients: with --wgrad beside they go to a second
+    # stream (lower priority than the data pass) and run beside the next layer's data pass on the SMs that pass leaves
+    # idle; the step ends when both streams are done.
+    w_stream = torch.cuda.Stream() if args.wgrad == "beside" else None
+
     def step_eager(s, freeze):
         if group:
             group_fwd(group, s, freeze)
         for L in singles:
             fwd(L, L["sets"][s], freeze)
+        cur_s = torch.cuda.current_stream()
         for L in reversed(singles):
-            bwd(L, L["sets"][s], freeze)
+            if w_stream is None:
+                bwd(L, L["sets"][s], freeze)
+                continue
+            bwd_data(L, L["sets"][s], freeze)
+            w_stream.wait_stream(cur_s)
+            with torch.cuda.stream(w_stream):
+                bwd_weights(L, L["sets"][s], freeze)
         if group:
             group_bwd(group, s, freeze)
+        if w_stream is not None:
+            cur_s.wait_stream(w_stream)
 
     masks = [b.LRD_FREEZE_U, b.LRD_FREEZE_V]
     # warm every (set, mask) once outside any capture: one-time kernel attribute set-up happens here
@@ -847,7 +872,7 @@ def main():
 
     graphs = {}
     if not args.no_graph:
-        side = torch.cuda.Stream()
+        side = torch.cuda.Stream(priority=-1)
         for s in range(S):
             for f in masks:
                 g = torch.cuda.CUDAGraph()
@@ -863,7 +888,7 @@ def main():
     cycle = 2 * S
     cycle_graph = None
     if graphs and not args.single_step_graphs:
-        side = torch.cuda.Stream()
+        side = torch.cuda.Stream(priority=-1)
         cycle_graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
             with torch.cuda.graph(cycle_graph, stream=side):
@@ -946,7 +971,7 @@ def main():
     if S > 1:
         hot_graph = None
         if cycle_graph is not None:              # the same cycle of 2 S steps, all on buffer set 0
-            side = torch.cuda.Stream()
+            side = torch.cuda.Stream(priority=-1)
             hot_graph = torch.cuda.CUDAGraph()
             with torch.cuda.stream(side):
                 with torch.cuda.graph(hot_graph, stream=side):
@@ -1136,6 +1161,8 @@ def main():
                                        "launch": "eager C-ABI calls" if args.no_graph else ("CUDA graph replay of the C-ABI calls, one graph per step" if args.single_step_graphs
                                                   else f"CUDA graph replay of the C-ABI calls, one graph per cycle of {cycle} steps (every buffer set under both masks)"),
                                        "path": args.path,
+                                       "weight_gradients": {"beside": "on a second stream beside the next layer's data pass (two-call backward), joined at the end of the step",
+                                                            "inline": "one backward call per layer"}[args.wgrad],
                                        "groups": {"qkv": "attn_q/k/v side by side in one group call, the other layers one call each",
                                                   "none": "one call per layer"}[args.groups]}),
                 "repeats": {"n": len(samples), "min_ms": samples[0] / args.steps, "max_ms": samples[-1] / args.steps, "reported": "median"},

@@ -233,6 +233,20 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
                             const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                             lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The backward pass in two calls, for callers that schedule the weight gradients themselves (Section 2.2: with one
+ * factor frozen only the other one's product is left, and nothing later in the backward pass of the network waits
+ * for it): lrd_linear_bwd_data forms dZ = dY U and dX = dZ V^T (dX nullable) and leaves dZ in the workspace when V is
+ * unfrozen; lrd_linear_bwd_weights forms the unfrozen factor's gradients (dU = dY^T Z_save with dbias, dV = X^T dZ),
+ * zero-fills the frozen one's buffers, and may run on another stream beside the next layer's data call.  When V is
+ * unfrozen the weights call reads the dZ its layer's data call left in the SAME workspace: order it after that call
+ * (same stream, or an event) and let nothing else use the workspace in between.  Together the two calls do exactly
+ * what lrd_linear_bwd does (same kernels, same bits); arguments, layouts and errors as there. */
+lrd_status_t lrd_linear_bwd_data(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
+                                 lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
+lrd_status_t lrd_linear_bwd_weights(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,
+                                    void* dV, void* dbias, lrd_freeze_t freeze, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream);
+
 /* Backward with gradient accumulation: as lrd_linear_bwd, but the unfrozen factor's dU, dbias and dV are ADDED to
  * what the buffers hold (gradient accumulation over micro-batches) instead of overwritten; dX is overwritten as
  * usual.  A frozen factor's gradient buffers are not touched at all (its gradient is zero), and may be NULL.

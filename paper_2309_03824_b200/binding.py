@@ -29,7 +29,7 @@ EXPORTS = [
     "lrd_rank_quantize", "lrd_freeze_for_epoch", "lrd_tucker_freeze_for_epoch", "lrd_linear_bwd_plan",
     "lrd_status_string", "lrd_launch_count", "lrd_set_path", "lrd_check_device_status", "lrd_linear_workspace_bytes",
     "lrd_tucker2_workspace_bytes", "lrd_dense_workspace_bytes", "lrd_linear_fwd", "lrd_linear_bwd",
-    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_selftest_wait_timeout", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_rank_multiple", "lrd_svd_rank", "lrd_tucker_rank", "lrd_tucker_rank_min", "lrd_conv3x3_workspace_bytes", "lrd_conv3x3_fwd", "lrd_conv3x3_bwd", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate",
+    "lrd_dense_fwd", "lrd_dense_bwd", "lrd_tucker2_fwd", "lrd_tucker2_bwd", "lrd_bias_grad_noalloc", "lrd_chain_tuning", "lrd_chain_pair_tuning", "lrd_selftest_wait_timeout", "lrd_gemm_tuning", "lrd_tucker2_overlap", "lrd_rank_search", "lrd_rank_multiple", "lrd_svd_rank", "lrd_tucker_rank", "lrd_tucker_rank_min", "lrd_conv3x3_workspace_bytes", "lrd_conv3x3_fwd", "lrd_conv3x3_bwd", "lrd_linear_group_fwd", "lrd_linear_group_bwd", "lrd_linear_bwd_accumulate", "lrd_linear_bwd_data", "lrd_linear_bwd_weights",
 ]
 
 
@@ -100,6 +100,10 @@ _lib.lrd_linear_fwd.restype = _int
 _lib.lrd_linear_fwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 6 + [_int, _vp, _sz, _vp]
 _lib.lrd_linear_bwd.restype = _int
 _lib.lrd_linear_bwd.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 9 + [_int, _vp, _sz, _vp]
+_lib.lrd_linear_bwd_data.restype = _int
+_lib.lrd_linear_bwd_data.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 4 + [_int, _vp, _sz, _vp]
+_lib.lrd_linear_bwd_weights.restype = _int
+_lib.lrd_linear_bwd_weights.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 6 + [_int, _vp, _sz, _vp]
 _lib.lrd_linear_bwd_accumulate.restype = _int
 _lib.lrd_linear_bwd_accumulate.argtypes = [C.POINTER(lrd_linear_desc_t)] + [_vp] * 9 + [_int, _vp, _sz, _vp]
 _lib.lrd_dense_fwd.restype = _int
@@ -280,6 +284,23 @@ def lrd_linear_bwd(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspa
     w, n = _ws(workspace)
     st = _lib.lrd_linear_bwd(C.byref(desc), _ptr(dY), _ptr(X), _ptr(V), _ptr(U), _ptr(Z_save), _ptr(dX), _ptr(dU),
                              _ptr(dV), _ptr(dbias), freeze, w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_linear_bwd_data(desc, dY, V, U, dX, freeze, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_linear_bwd_data(C.byref(desc), _ptr(dY), _ptr(V), _ptr(U), _ptr(dX), freeze, w, n, _stream(stream))
+    if check:
+        _check(st)
+    return st
+
+
+def lrd_linear_bwd_weights(desc, dY, X, Z_save, dU, dV, dbias, freeze, workspace, stream=None, check=True):
+    w, n = _ws(workspace)
+    st = _lib.lrd_linear_bwd_weights(C.byref(desc), _ptr(dY), _ptr(X), _ptr(Z_save), _ptr(dU), _ptr(dV), _ptr(dbias), freeze, w, n,
+                                     _stream(stream))
     if check:
         _check(st)
     return st

@@ -492,14 +492,17 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
                                   const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                                   lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, cudaStream_t s,
                                   cudaStream_t side, cudaEvent_t side_done, int sm_share, bool check_only = false,
-                                  bool data_done = false) {
+                                  int parts = 3) {
+    // parts: 1 = the data half (dZ, dX), 2 = the weight-gradient half (it reads the dZ the data half left in the
+    // workspace when V is unfrozen), 3 = both
+    const bool do_data = (parts & 1) != 0, do_w = (parts & 2) != 0;
     Linear L;
     LRD_TRY(parse_linear(desc, &L, false));
     const uint32_t plan = lrd_linear_bwd_plan(freeze);
     if (!plan) return LRD_ERR_INVALID_ARG;
-    if (!dY || !V || !U) return LRD_ERR_INVALID_ARG;
-    if ((plan & LRD_PLAN_NEEDS_Z) && (!Z_save || !dU)) return LRD_ERR_INVALID_ARG;
-    if ((plan & LRD_PLAN_NEEDS_X) && (!X || !dV)) return LRD_ERR_INVALID_ARG;
+    if (!dY || (do_data && (!V || !U))) return LRD_ERR_INVALID_ARG;
+    if (do_w && (plan & LRD_PLAN_NEEDS_Z) && (!Z_save || !dU)) return LRD_ERR_INVALID_ARG;
+    if (do_w && (plan & LRD_PLAN_NEEDS_X) && (!X || !dV)) return LRD_ERR_INVALID_ARG;
     const void* ptrs[] = {dY, X, V, U, Z_save, dX, dU, dV, dbias};
     for (const void* p : ptrs)
         if (p && !elem_aligned(p, L.dt)) return LRD_ERR_ALIGNMENT;
@@ -508,29 +511,31 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
     if (check_only) return LRD_OK;
 
     // frozen factor: no product is launched; a gradient buffer the caller passed reads as zero
-    if (!(plan & LRD_PLAN_DU)) {
+    if (do_w && !(plan & LRD_PLAN_DU)) {
         LRD_TRY(zero_fill(dU, L.N, L.r, L.ldu, L.dt, s));
         LRD_TRY(zero_fill(dbias, 1, L.N, L.N, L.dt, s));
     }
-    if (!(plan & LRD_PLAN_DV)) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
+    if (do_w && !(plan & LRD_PLAN_DV)) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
     if (L.M == 0) {                      // no tokens: the unfrozen gradients are sums over nothing
-        if (plan & LRD_PLAN_DU) { LRD_TRY(zero_fill(dU, L.N, L.r, L.ldu, L.dt, s)); LRD_TRY(zero_fill(dbias, 1, L.N, L.N, L.dt, s)); }
-        if (plan & LRD_PLAN_DV) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
+        if (do_w && (plan & LRD_PLAN_DU)) { LRD_TRY(zero_fill(dU, L.N, L.r, L.ldu, L.dt, s)); LRD_TRY(zero_fill(dbias, 1, L.N, L.N, L.dt, s)); }
+        if (do_w && (plan & LRD_PLAN_DV)) LRD_TRY(zero_fill(dV, L.K, L.r, L.ldv, L.dt, s));
         return LRD_OK;
     }
 
-    if (needs_repack(L) && g_path.load() != LRD_PATH_GENERAL && L.ldx % 8 == 0 && L.ldy % 8 == 0 && !data_done) {
+    if (needs_repack(L) && g_path.load() != LRD_PATH_GENERAL && L.ldx % 8 == 0 && L.ldy % 8 == 0) {
         const lrd_linear_desc_t q = padded_desc(*desc, L);
         const size_t inner = lrd_linear_workspace_bytes(&q, freeze, 1);
         const RepackLayout o = repack_layout(L, inner);
         uint8_t* w = (uint8_t*)workspace;
-        const bool du = (plan & LRD_PLAN_DU) != 0, dv = (plan & LRD_PLAN_DV) != 0;
-        LRD_TRY(copy2d_bf16(w + o.Vp, q.r, V, L.ldv, L.K, L.r, q.r, s));
-        LRD_TRY(copy2d_bf16(w + o.Up, q.r, U, L.ldu, L.N, L.r, q.r, s));
+        const bool du = do_w && (plan & LRD_PLAN_DU) != 0, dv = do_w && (plan & LRD_PLAN_DV) != 0;
+        if (do_data) {
+            LRD_TRY(copy2d_bf16(w + o.Vp, q.r, V, L.ldv, L.K, L.r, q.r, s));
+            LRD_TRY(copy2d_bf16(w + o.Up, q.r, U, L.ldu, L.N, L.r, q.r, s));
+        }
         if (du) LRD_TRY(copy2d_bf16(w + o.Zp, q.r, Z_save, L.ldz, L.M, L.r, q.r, s));
         // the frozen factor's buffers were zero-filled above; the padded call gets none for them
-        LRD_TRY(linear_bwd_on(&q, dY, X, w + o.Vp, w + o.Up, du ? w + o.Zp : nullptr, dX, du ? w + o.dUp : nullptr, dv ? w + o.dVp : nullptr,
-                              du ? dbias : nullptr, freeze, w, inner, s, nullptr, nullptr, sm_share));
+        LRD_TRY(linear_bwd_on(&q, dY, X, w + o.Vp, w + o.Up, w + o.Zp, dX, w + o.dUp, w + o.dVp, du ? dbias : nullptr, freeze, w, inner, s,
+                              nullptr, nullptr, sm_share, false, parts));
         if (du) LRD_TRY(copy2d_bf16(dU, L.ldu, w + o.dUp, q.r, L.N, L.r, L.r, s));
         if (dv) LRD_TRY(copy2d_bf16(dV, L.ldv, w + o.dVp, q.r, L.K, L.r, L.r, s));
         return LRD_OK;
@@ -541,7 +546,7 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
     const size_t partial_bytes = workspace_bytes - linear_z_bytes(L);
     const bool need_dz_in_memory = (plan & LRD_PLAN_DV) != 0;
 
-    bool chained = data_done;            // a group has already run this layer's data chain (dX, and dZ where needed)
+    bool chained = !do_data;             // the data half (dX, and dZ where needed) has run already, or runs in a later call
     const int path = g_path.load();
     if (!chained && dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED)) {
         const ChainArgs c = bwd_chain_args(L, dY, V, U, dX, need_dz_in_memory ? dZ : nullptr, sm_share);
@@ -555,7 +560,7 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
         if (dX)
             LRD_TRY(run_gemm(gemm(L.M, L.K, L.r, dZ, L.r, false, V, L.ldv, false, dX, L.ldx, nullptr, L.dt), false, nullptr, 0, s));
     }
-    if (plan & LRD_PLAN_DU) {
+    if (do_w && (plan & LRD_PLAN_DU)) {
         GemmArgs gu = gemm(L.N, L.r, L.M, dY, L.ldy, true, Z_save, L.ldz, true, dU, L.ldu, nullptr, L.dt);
         bool db_done = false;
         if (dbias && g_path.load() != LRD_PATH_GENERAL) {      // db rides on the dU product (A = dY): no second pass over dY
@@ -569,10 +574,23 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
             if (cudaEventRecord(side_done, side) != cudaSuccess || cudaStreamWaitEvent(s, side_done, 0) != cudaSuccess) return LRD_ERR_CUDA;
         }
     }
-    if (plan & LRD_PLAN_DV)
+    if (do_w && (plan & LRD_PLAN_DV))
         LRD_TRY(run_gemm(gemm(L.K, L.r, L.M, X, L.ldx, true, dZ, L.r, true, dV, L.ldv, nullptr, L.dt), true, partials,
                          partial_bytes, s));
     return LRD_OK;
+}
+
+lrd_status_t lrd_linear_bwd_data(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
+                                 lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return linear_bwd_on(desc, dY, nullptr, V, U, nullptr, dX, nullptr, nullptr, nullptr, freeze, workspace, workspace_bytes,
+                         (cudaStream_t)cuda_stream, nullptr, nullptr, 0, false, 1);
+}
+
+lrd_status_t lrd_linear_bwd_weights(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,
+                                    void* dV, void* dbias, lrd_freeze_t freeze, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+    return linear_bwd_on(desc, dY, X, nullptr, nullptr, Z_save, nullptr, dU, dV, dbias, freeze, workspace, workspace_bytes,
+                         (cudaStream_t)cuda_stream, nullptr, nullptr, 0, false, 2);
 }
 
 lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
@@ -705,7 +723,7 @@ lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const v
         if (sd && cudaStreamWaitEvent(sd, ss->fork, 0) != cudaSuccess) { st = LRD_ERR_CUDA; continue; }
         const lrd_status_t sti = linear_bwd_on(&descs[i], dY[i], at(X, i), V[i], U[i], at(Z_save, i), at_w(dX, i), at_w(dU, i),
                                                at_w(dV, i), at_w(dbias, i), freeze, workspace[i], workspace_bytes[i], si, sd,
-                                               ss->aux_done[i], share, false, data_done);
+                                               ss->aux_done[i], share, false, data_done ? 2 : 3);
         if (sti != LRD_OK) st = sti;
         if (sd && !stream_after(s, sd, ss->aux_done[i])) st = LRD_ERR_CUDA;
         if (i > 0 && !stream_after(s, si, ss->join[i - 1])) st = LRD_ERR_CUDA;

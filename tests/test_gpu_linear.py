@@ -92,6 +92,36 @@ def test_odd_factor_strides_leave_the_padding_alone():
         assert (got[:, w:] == 3.0).all()                      # columns past the rank are never written
 
 
+@pytest.mark.parametrize("shape", [(520, 264, 328, 64), (640, 768, 768, 192), (300, 200, 136, 33), (384, 3072, 768, 384)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_backward_in_two_calls_on_two_streams_gives_the_bits_of_one_call(shape, freeze):
+    """The data half on one stream, the weight-gradient half on another (ordered by an event, as a caller that runs the
+    weight gradients beside the next layer's data call would): same kernels, so the same bits as lrd_linear_bwd."""
+    M, K, N, r = shape
+    case = wl.random_factor_case(M, K, N, r, "bf16", 380 + M)
+    one = run_linear(case, freeze)
+    code, tdt = DT["bf16"]
+    X, V, U, bias, dY = (dev(case[k], "bf16") for k in ("X", "V", "U", "b", "dY"))
+    desc = b.linear_desc(M, K, N, r, code)
+    ws = workspace(max(b.lrd_linear_workspace_bytes(desc, freeze, 0), b.lrd_linear_workspace_bytes(desc, freeze, 1)))
+    Z = one["Z"]
+    nan = float("nan")
+    dX, dU, dV, db = (torch.full(sh, nan, dtype=tdt, device="cuda") for sh in ((M, K), (N, r), (K, r), (N,)))
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(main):
+        b.lrd_linear_bwd_data(desc, dY, V, U, dX, freeze, ws)
+        ev = torch.cuda.Event()
+        ev.record(main)
+    with torch.cuda.stream(side):
+        side.wait_event(ev)
+        b.lrd_linear_bwd_weights(desc, dY, None if freeze == b.LRD_FREEZE_V else X, Z, dU, dV, db, freeze, ws)
+    torch.cuda.synchronize()
+    assert b.lrd_check_device_status() == b.LRD_OK
+    for name, got in (("dX", dX), ("dU", dU), ("dV", dV), ("db", db)):
+        assert torch.equal(got, one[name]), name
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_once():
     """The self-test block waits on a barrier nothing arrives at; its wait gives up at the limit every pipeline wait
     has, the status check reports LRD_ERR_TIMEOUT exactly once, and the library keeps working afterwards."""

@@ -597,7 +597,7 @@ static SplitPlan pick_split(int64_t M, int64_t N, int64_t K, bool ones) {
             if (bn % (8 * S)) continue;
             if (tiles > max_active_clusters(S) || S > kb) continue;    // one wave: a second wave would double the time
             const double per_block = (double)((kb + S - 1) / S) * (A_STAGE_BYTES + bn * BK * 2.0);
-            const double t = std::max(per_block / 110e9, per_block * (double)(tiles * S) / 16e12) + 2e-6 * bn / 192.0;
+            const double t = std::max(per_block / 110e9, per_block * (double)(tiles * S) / 11.5e12) + 2e-6 * bn / 192.0;
             if (t < best_t) { best_t = t; best.bn = bn; best.cluster = S; best.global = 1; }
             break;                                                // the largest feasible cluster for this width
         }

@@ -94,19 +94,35 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(int64_t M, int64_t N, int
     const int64_t m0 = (int64_t)blockIdx.y * TM, n0 = (int64_t)blockIdx.x * TN;
     const int tx = t % 16, ty = t / 16;  // thread computes rows ty*4.., cols tx*4..
     float acc[4][4] = {};
-    for (int64_t k0 = 0; k0 < K; k0 += TK) {
+    // The next tile's elements are fetched into registers before the current tile is multiplied: their global-memory
+    // latency then runs beside the arithmetic instead of in front of it (the order of the additions is unchanged).
+    float ra[4], rb[4];
+    auto fetch = [&](int64_t k0) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             int mm, kk;
             if (la.k_fastest()) { mm = t / 16 + 16 * i; kk = t % 16; } else { kk = t / 64 + 4 * i; mm = t % 64; }
             const int64_t m = m0 + mm, k = k0 + kk;
-            As[kk][mm] = (m < M && k < K) ? la(m, k) : 0.f;
+            ra[i] = (m < M && k < K) ? la(m, k) : 0.f;
             int nn;
             if (lb.k_fastest()) { nn = t / 16 + 16 * i; kk = t % 16; } else { kk = t / 64 + 4 * i; nn = t % 64; }
             const int64_t n = n0 + nn, kb = k0 + kk;
-            Bs[kk][nn] = (n < N && kb < K) ? lb(kb, n) : 0.f;
+            rb[i] = (n < N && kb < K) ? lb(kb, n) : 0.f;
+        }
+    };
+    fetch(0);
+    for (int64_t k0 = 0; k0 < K; k0 += TK) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int mm, kk;
+            if (la.k_fastest()) { mm = t / 16 + 16 * i; kk = t % 16; } else { kk = t / 64 + 4 * i; mm = t % 64; }
+            As[kk][mm] = ra[i];
+            int nn;
+            if (lb.k_fastest()) { nn = t / 16 + 16 * i; kk = t % 16; } else { kk = t / 64 + 4 * i; nn = t % 64; }
+            Bs[kk][nn] = rb[i];
         }
         __syncthreads();
+        if (k0 + TK < K) fetch(k0 + TK);
 #pragma unroll
         for (int kk = 0; kk < TK; ++kk) {
             float a[4], b[4];

@@ -214,6 +214,13 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         uint32_t slices_ready = 1u << c;
         const uint32_t idesc2 = idesc_bf16(p.BN2, false, false);
         const uint64_t t_desc0 = smem_desc(t_base, 0, 8u * t_sw, t_sw);
+        // T's descriptor for k-step kk of k-block kb is t_desc0 + kb * tk_stride + tk_off[kk] (16-byte units): what the
+        // issuing thread computes per MMA is kept to one add (its instructions are what paces a stage of four MMAs)
+        const uint32_t tk_stride = ((4u >> p.t_steps_lg) * t_atom_bytes) >> 4;
+        uint32_t tk_off[4];
+#pragma unroll
+        for (uint32_t kk = 0; kk < 4; ++kk)
+            tk_off[kk] = (((kk >> p.t_steps_lg) * t_atom_bytes) + (kk & ((1u << p.t_steps_lg) - 1u)) * 32u) >> 4;
         s = 0;
         ph = 0;
         int i2 = 0;
@@ -239,11 +246,11 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
                 const uint32_t q_src = ring2_base + s * p.stage2_bytes;
                 const uint64_t bd = a_desc0 + ((q_src >> 4) & 0x3FFFu);
                 if (elect_one()) {
-                    for (int kk = 0; kk < nks; ++kk) {
-                        const uint32_t ks = (uint32_t)(kb * 4 + kk);      // 16-column step within T
-                        const uint64_t ad = t_desc0 + (((ks >> p.t_steps_lg) * t_atom_bytes + (ks & ((1u << p.t_steps_lg) - 1u)) * 32u) >> 4);
-                        mma_bf16_ss(d_tmem, ad, bd + 2u * kk, idesc2, (i > 0 || kk > 0) ? 1u : 0u);
-                    }
+                    const uint64_t adk = t_desc0 + (uint32_t)kb * tk_stride;
+                    const uint32_t acc = i > 0 ? 1u : 0u;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)                        // 16-column steps within T
+                        if (kk < nks) mma_bf16_ss(d_tmem, adk + tk_off[kk], bd + 2u * kk, idesc2, kk > 0 ? 1u : acc);
                     mma_commit(smem_u32(&empty2[s]));
                     if (i == p.kb2 - 1) mma_commit(smem_u32(&out_full[i2 & 1]));
                 }
@@ -478,9 +485,10 @@ bool make_plan(const ChainArgs& a, Plan* out) {
         const int64_t ring2 = ring1 - t_bytes - (int64_t)kStagingBytes;
         const uint32_t kb1_bytes = kInTileBytes + 128u * RS, kb2_bytes = (uint32_t)BN2 * 128u;
         if (ring2 < 2 * (int64_t)kb2_bytes) continue;
-        // phase 1: one k-block per stage (the finest pipeline); two for a short reduction, where the number of
-        // copies counts for more than the depth of the ring
-        int G1 = g_tune_G1 ? g_tune_G1 : (kb1 <= 16 ? 2 : 1);
+        // phase 1: two k-blocks per stage: what a stage costs the issuing threads beside its copies and MMAs (a wait,
+        // an election, a commit: some 250 cycles) is then spread over eight MMAs of r / C columns, which by
+        // themselves take 40-60 cycles each (measured: one per stage 21.9, two 20.2, three 22.0 us on 3072 -> 768)
+        int G1 = g_tune_G1 ? g_tune_G1 : 2;
         if (G1 > 4) G1 = 4;
         if (G1 > kb1) G1 = kb1;
         while (!g_tune_G1 && G1 > 1 && ring1 < 2 * (int64_t)G1 * kb1_bytes) --G1;   // a wide T buffer leaves room for single k-blocks only

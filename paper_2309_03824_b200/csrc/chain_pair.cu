@@ -573,7 +573,12 @@ bool chain_pair_preferred(const ChainArgs* layers, int n) {
     if (!chain_pair_eligible(layers, n)) return false;
     Plan pl;
     if (!make_plan(layers[0], n, &pl) || pl.NS2 < 3) return false;
-    return n > 1 || layers[0].K1 >= 2 * layers[0].N2;
+    // Measured against the chain on single blocks: pairs win for groups, where the first product dominates, where
+    // the single blocks' T buffer leaves fewer than three weight tiles in flight (r = 512), and at r >= 384 once
+    // there are more row tiles than clusters of four fit on the GPU (8192 tokens, 4096 x 4096: r = 384 59 against
+    // 64 us forward, r = 512 62 against 85; r = 256 stays on single blocks, 50 against 54).
+    const ChainArgs& a = layers[0];
+    return n > 1 || a.K1 >= 2 * a.N2 || (a.r > 384 && !chain_preferred(a)) || (a.r >= 384 && (a.M + 127) / 128 > 37);
 }
 
 lrd_status_t chain_pair_launch(const ChainArgs* layers, int n, cudaStream_t stream) {

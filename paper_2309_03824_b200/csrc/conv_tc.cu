@@ -142,14 +142,13 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
             if (!ok) break;
             tc_fence_after();
             const uint32_t a_src = smem_base + s * kStageBytes, b_src = a_src + kTile;
+            const int nks = min(4, (p.ka - (it % nkc) * 64 + 15) / 16);      // 16-channel steps past ka hold zeros: not issued
             if (elect_one()) {
+                const uint64_t ad0 = smem_desc_sw128(a_src, 0, 1024);
+                const uint64_t bd0 = DGRAD ? smem_desc_sw128(b_src, 8192, 1024) : smem_desc_sw128(b_src, 0, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ad = smem_desc_sw128(a_src + kk * 32, 0, 1024);
-                    const uint64_t bd = DGRAD ? smem_desc_sw128(b_src + kk * 2048, 8192, 1024)
-                                              : smem_desc_sw128(b_src + kk * 32, 0, 1024);
-                    mma_bf16_ss(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < 4; ++kk)                               // the k-step moves the start address only
+                    if (kk < nks) mma_bf16_ss(tmem_base, ad0 + 2u * kk, bd0 + (DGRAD ? 128u : 2u) * kk, idesc, (it > 0 || kk > 0) ? 1u : 0u);
                 mma_commit(smem_u32(&empty_bar[s]));
             }
             __syncwarp();

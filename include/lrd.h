@@ -87,7 +87,11 @@ typedef struct {
 
 typedef struct {
     int64_t B, H, W, C, S, r1, r2;  /* NHWC activations [B][H][W][C] -> [B][H][W][S] */
-    int64_t k, stride, pad;         /* only k = 3, stride = 1, pad = 1 */
+    int64_t k, stride, pad;         /* k x k core: k odd, 1..7; stride 1 or 2 (on the core); pad = (k - 1) / 2.
+                                     * The output is [B][Ho][Wo][S] with Ho = (H - 1) / stride + 1, Wo likewise.
+                                     * k = 3, stride = 1 runs the core on the tensor-core kernels (bf16, shapes
+                                     * permitting); every other geometry runs it on the general fp32-FMA kernels.
+                                     * Anything else: LRD_ERR_UNSUPPORTED. */
     int32_t dtype;
 } lrd_tucker2_desc_t;
 
@@ -326,20 +330,21 @@ lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const 
 lrd_status_t lrd_bias_grad_noalloc(const void* dY, int64_t ldy, int64_t M, int64_t N, void* dbias,
                                    lrd_dtype_t dtype, void* cuda_stream);
 
-/* ---- Tucker-2 decomposed 3x3 convolution (Eq. 4, Fig. 1) -------------------------------- */
+/* ---- Tucker-2 decomposed k x k convolution (Eq. 4, Fig. 1) -------------------------------- */
 
-/* Forward: Z1 = X A (1x1, C -> r1); Z2 = conv3x3(Z1, G) (cross-correlation, stride 1, zero pad 1,
- * r1 -> r2); Y = Z2 Bm^T + bias (1x1, r2 -> S).  NHWC: X[B][H][W][C], Y[B][H][W][S]; A[C x r1],
- * G[r2][3][3][r1], Bm[S x r2], bias[S] or NULL.
+/* Forward: Z1 = X A (1x1, C -> r1); Z2 = conv(Z1, G) (cross-correlation, k x k, the layer's stride, zero pad
+ * (k - 1) / 2, r1 -> r2: output pixel (ho, wo) reads input pixels (ho stride + kh - pad, wo stride + kw - pad));
+ * Y = Z2 Bm^T + bias (1x1, r2 -> S).  NHWC: X[B][H][W][C], Y[B][Ho][Wo][S]; A[C x r1], G[r2][k][k][r1],
+ * Bm[S x r2], bias[S] or NULL.
  *   Z1_save[B][H][W][r1]: required unless freeze == LRD_TK_FREEZE_CORE (then must be NULL);
- *   Z2_save[B][H][W][r2]: required unless freeze == LRD_TK_FREEZE_FACTORS (then must be NULL). */
+ *   Z2_save[B][Ho][Wo][r2]: required unless freeze == LRD_TK_FREEZE_FACTORS (then must be NULL). */
 lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, const void* A, const void* G,
                              const void* Bm, const void* bias, void* Y, void* Z1_save, void* Z2_save,
                              lrd_tucker_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Backward: dZ2 = dY Bm; dZ1 = conv3x3^T(dZ2, G); dX = dZ1 A^T (NULL skips);
+/* Backward (dY[B][Ho][Wo][S]): dZ2 = dY Bm; dZ1 = conv^T(dZ2, G); dX[B][H][W][C] = dZ1 A^T (NULL skips);
  *   factors not frozen: dB[S x r2] = dY^T Z2_save, dA[C x r1] = X^T dZ1, dbias = column sums of dY;
- *   core not frozen:    dG[o][kh][kw][i] = sum_p dZ2[p][o] Z1_save[p shifted by (kh-1, kw-1)][i].
+ *   core not frozen:    dG[o][kh][kw][i] = sum_p dZ2[p][o] Z1_save[p stride + (kh, kw) - pad][i] (p: output pixels).
  * Frozen groups: product not launched, non-NULL gradient pointers are zero-filled. */
 lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, const void* X, const void* A,
                              const void* G, const void* Bm, const void* Z1_save, const void* Z2_save, void* dX,

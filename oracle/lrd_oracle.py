@@ -257,24 +257,26 @@ def tucker2_reconstruct(A, G, Bm):
     return np.einsum("ohwi,ci,so->schw", _f64(G), _f64(A), _f64(Bm))
 
 
-def conv2d_nhwc_fwd(X, Wk, pad):
-    """Cross-correlation, stride 1, zero padding.  X[B][H][W][Ci], Wk[Co][k][k][Ci] ->
-    Y[B][H][W][Co]  (pad = (k-1)/2 keeps the spatial size)."""
+def conv2d_nhwc_fwd(X, Wk, pad, stride=1):
+    """Cross-correlation with zero padding.  X[B][H][W][Ci], Wk[Co][k][k][Ci] -> Y[B][Ho][Wo][Co] with
+    Y[b,ho,wo,o] = sum_{kh,kw,i} Xpadded[b, ho*stride + kh, wo*stride + kw, i] Wk[o,kh,kw,i] and
+    Ho = (H + 2 pad - k) // stride + 1  (stride 1 and pad = (k-1)/2 keep the spatial size)."""
     X, Wk = _f64(X), _f64(Wk)
     B, H, Wd, Ci = X.shape
     Co, k, _, _ = Wk.shape
-    Ho, Wo = H + 2 * pad - k + 1, Wd + 2 * pad - k + 1
+    Ho, Wo = (H + 2 * pad - k) // stride + 1, (Wd + 2 * pad - k) // stride + 1
     Xp = np.zeros((B, H + 2 * pad, Wd + 2 * pad, Ci))
     Xp[:, pad:pad + H, pad:pad + Wd, :] = X
     Y = np.zeros((B, Ho, Wo, Co))
     for kh in range(k):
         for kw in range(k):
-            Y += Xp[:, kh:kh + Ho, kw:kw + Wo, :] @ Wk[:, kh, kw, :].T
+            Y += Xp[:, kh:kh + (Ho - 1) * stride + 1:stride, kw:kw + (Wo - 1) * stride + 1:stride, :] @ Wk[:, kh, kw, :].T
     return Y
 
 
-def conv2d_nhwc_bwd_data(dY, Wk, pad, in_hw):
-    """dX[b,h,w,i] = sum_{o,kh,kw} dY[b, h+pad-kh, w+pad-kw, o] Wk[o,kh,kw,i]."""
+def conv2d_nhwc_bwd_data(dY, Wk, pad, in_hw, stride=1):
+    """dXpadded[b, ho*stride + kh, wo*stride + kw, i] += dY[b,ho,wo,o] Wk[o,kh,kw,i] over all (ho, wo, kh, kw, o);
+    dX is its interior (for stride 1: dX[b,h,w,i] = sum_{o,kh,kw} dY[b, h+pad-kh, w+pad-kw, o] Wk[o,kh,kw,i])."""
     dY, Wk = _f64(dY), _f64(Wk)
     B, Ho, Wo, Co = dY.shape
     _, k, _, Ci = Wk.shape
@@ -282,12 +284,12 @@ def conv2d_nhwc_bwd_data(dY, Wk, pad, in_hw):
     dXp = np.zeros((B, H + 2 * pad, Wd + 2 * pad, Ci))
     for kh in range(k):
         for kw in range(k):
-            dXp[:, kh:kh + Ho, kw:kw + Wo, :] += dY @ Wk[:, kh, kw, :]
+            dXp[:, kh:kh + (Ho - 1) * stride + 1:stride, kw:kw + (Wo - 1) * stride + 1:stride, :] += dY @ Wk[:, kh, kw, :]
     return dXp[:, pad:pad + H, pad:pad + Wd, :]
 
 
-def conv2d_nhwc_bwd_filter(dY, X, k, pad):
-    """dWk[o,kh,kw,i] = sum_{b,h,w} dY[b,h,w,o] Xpadded[b,h+kh,w+kw,i]."""
+def conv2d_nhwc_bwd_filter(dY, X, k, pad, stride=1):
+    """dWk[o,kh,kw,i] = sum_{b,ho,wo} dY[b,ho,wo,o] Xpadded[b, ho*stride + kh, wo*stride + kw, i]."""
     dY, X = _f64(dY), _f64(X)
     B, H, Wd, Ci = X.shape
     _, Ho, Wo, Co = dY.shape
@@ -297,24 +299,24 @@ def conv2d_nhwc_bwd_filter(dY, X, k, pad):
     dYm = dY.reshape(-1, Co)
     for kh in range(k):
         for kw in range(k):
-            dW[:, kh, kw, :] = dYm.T @ Xp[:, kh:kh + Ho, kw:kw + Wo, :].reshape(-1, Ci)
+            dW[:, kh, kw, :] = dYm.T @ Xp[:, kh:kh + (Ho - 1) * stride + 1:stride, kw:kw + (Wo - 1) * stride + 1:stride, :].reshape(-1, Ci)
     return dW
 
 
-def tucker2_fwd(X, A, G, Bm, bias=None):
-    """1x1 (C -> r1), k x k core (r1 -> r2, stride 1, pad (k-1)/2), 1x1 (r2 -> S).
-    X[B][H][W][C] -> (Z1[B][H][W][r1], Z2[B][H][W][r2], Y[B][H][W][S])."""
+def tucker2_fwd(X, A, G, Bm, bias=None, stride=1):
+    """1x1 (C -> r1), k x k core (r1 -> r2, pad (k-1)/2; the layer's stride sits on the core), 1x1 (r2 -> S).
+    X[B][H][W][C] -> (Z1[B][H][W][r1], Z2[B][Ho][Wo][r2], Y[B][Ho][Wo][S])."""
     X, A, G, Bm = _f64(X), _f64(A), _f64(G), _f64(Bm)
     k = G.shape[1]
     Z1 = X @ A
-    Z2 = conv2d_nhwc_fwd(Z1, G, (k - 1) // 2)
+    Z2 = conv2d_nhwc_fwd(Z1, G, (k - 1) // 2, stride)
     Y = Z2 @ Bm.T
     if bias is not None:
         Y = Y + _f64(bias)
     return Z1, Z2, Y
 
 
-def tucker2_bwd(dY, X, A, G, Bm, Z1, Z2, freeze=TK_FREEZE_NONE):
+def tucker2_bwd(dY, X, A, G, Bm, Z1, Z2, freeze=TK_FREEZE_NONE, stride=1):
     """Chain rule through the three convolutions.  Data gradients always flow; a frozen
     group's weight gradients are exactly zero.  The bias belongs to the last 1x1 factor.
     Returns dict(dX, dA, dG, dB, db)."""
@@ -323,7 +325,7 @@ def tucker2_bwd(dY, X, A, G, Bm, Z1, Z2, freeze=TK_FREEZE_NONE):
     pad = (k - 1) // 2
     S, C = Bm.shape[0], A.shape[0]
     dZ2 = dY @ Bm
-    dZ1 = conv2d_nhwc_bwd_data(dZ2, G, pad, X.shape[1:3])
+    dZ1 = conv2d_nhwc_bwd_data(dZ2, G, pad, X.shape[1:3], stride)
     out = {"dX": dZ1 @ A.T}
     if freeze == TK_FREEZE_FACTORS:
         out["dA"], out["dB"], out["db"] = np.zeros_like(A), np.zeros_like(Bm), np.zeros(S)
@@ -331,7 +333,7 @@ def tucker2_bwd(dY, X, A, G, Bm, Z1, Z2, freeze=TK_FREEZE_NONE):
         out["dA"] = X.reshape(-1, C).T @ dZ1.reshape(-1, A.shape[1])
         out["dB"] = dY.reshape(-1, S).T @ _f64(Z2).reshape(-1, Bm.shape[1])
         out["db"] = dY.reshape(-1, S).sum(axis=0)
-    out["dG"] = np.zeros_like(G) if freeze == TK_FREEZE_CORE else conv2d_nhwc_bwd_filter(dZ2, _f64(Z1), k, pad)
+    out["dG"] = np.zeros_like(G) if freeze == TK_FREEZE_CORE else conv2d_nhwc_bwd_filter(dZ2, _f64(Z1), k, pad, stride)
     return out
 
 

@@ -1,5 +1,6 @@
-// Tucker-2 decomposed 3x3 convolution (NHWC): 1x1 product, 3x3 core, 1x1 product, and the
-// backward pass through them under a freeze mask.
+// Tucker-2 decomposed k x k convolution (NHWC): 1x1 product, k x k core (which carries the layer's stride), 1x1
+// product, and the backward pass through them under a freeze mask.  The 3 x 3, stride-1 core runs on the
+// tensor-core kernels where the shape allows; every other geometry runs the core on the general kernels.
 #include "conv.cuh"
 
 #include "streams.cuh"
@@ -9,19 +10,28 @@ namespace lrd {
 namespace {
 
 struct Tk {
-    int64_t B, H, W, C, S, r1, r2, P;
+    int64_t B, H, W, C, S, r1, r2;
+    int64_t P;              // input pixels B H W (rows of X, Z1, dZ1, dX)
+    int64_t Po;             // output pixels B Ho Wo (rows of Z2, Y, dY, dZ2)
+    int64_t taps;           // k * k
+    ConvGeom g;
+    bool plain;             // 3 x 3, stride 1: the geometry the tensor-core core kernels take
     lrd_dtype_t dt;
 };
 
 Tk parse(const lrd_tucker2_desc_t* d) {
     Tk t;
     t.B = d->B; t.H = d->H; t.W = d->W; t.C = d->C; t.S = d->S; t.r1 = d->r1; t.r2 = d->r2;
+    t.g = conv_geom(d->H, d->W, d->k, d->stride);
     t.P = d->B * d->H * d->W;
+    t.Po = d->B * t.g.Ho * t.g.Wo;
+    t.taps = d->k * d->k;
+    t.plain = d->k == 3 && d->stride == 1;
     t.dt = (lrd_dtype_t)d->dtype;
     return t;
 }
 
-size_t act_bytes(const Tk& t, int64_t ch) { return align_up((size_t)(t.P > 0 ? t.P : 1) * ch * elem_size(t.dt), 256); }
+size_t act_bytes(const Tk& t, int64_t pixels, int64_t ch) { return align_up((size_t)(pixels > 0 ? pixels : 1) * ch * elem_size(t.dt), 256); }
 
 // Scratch of the three weight-gradient launches of the backward pass, one region each: they may run side by side.
 struct Scratch { size_t dB, dA, filter; };
@@ -29,12 +39,12 @@ struct Scratch { size_t dB, dA, filter; };
 Scratch split_regions(const Tk& t) {
     Scratch r{0, 0, 0};
     if (t.P < 1) return r;
-    r.dB = colsum_scratch_bytes(t.P, t.S);
+    r.dB = colsum_scratch_bytes(t.Po, t.S);
     if (t.dt == LRD_BF16) {
-        const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.P);
+        const size_t a = tc_split_workspace_bytes(t.S, t.r2, t.Po);
         r.dB = r.dB > a ? r.dB : a;
         r.dA = tc_split_workspace_bytes(t.C, t.r1, t.P);
-        r.filter = tc_conv_filter_scratch_bytes(t.B, t.H, t.W, t.r1, t.r2);
+        if (t.plain) r.filter = tc_conv_filter_scratch_bytes(t.B, t.H, t.W, t.r1, t.r2);
     }
     r.dB = align_up(r.dB, 256); r.dA = align_up(r.dA, 256); r.filter = align_up(r.filter, 256);
     return r;
@@ -51,7 +61,7 @@ bool g_tucker_overlap = true;
 // layer, the factors -- small -- are copied into the workspace with the ranks rounded up to multiples of 16 and
 // zeros in the padding, the layer runs on the tensor-core kernels at the padded ranks, and Z1 / Z2 / dA / dG / dB
 // are copied between the caller's packed layout and padded buffers.
-bool needs_repack(const Tk& t) { return t.dt == LRD_BF16 && (t.r1 % 8 || t.r2 % 8) && t.C % 8 == 0 && t.S % 8 == 0; }
+bool needs_repack(const Tk& t) { return t.plain && t.dt == LRD_BF16 && (t.r1 % 8 || t.r2 % 8) && t.C % 8 == 0 && t.S % 8 == 0; }
 int64_t pad16(int64_t r) { return (r + 15) / 16 * 16; }
 lrd_tucker2_desc_t padded_desc(const lrd_tucker2_desc_t& d) {
     lrd_tucker2_desc_t q = d;
@@ -86,7 +96,8 @@ lrd_status_t tucker2_check(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t free
     if (d->B < 0 || d->H < 1 || d->W < 1 || d->C < 1 || d->S < 1) return LRD_ERR_INVALID_ARG;
     if (d->dtype != LRD_F32 && d->dtype != LRD_BF16) return LRD_ERR_INVALID_ARG;
     if (d->r1 < 1 || d->r2 < 1 || d->r1 > d->C || d->r2 > d->S) return LRD_ERR_BAD_RANK;
-    if (d->k != 3 || d->stride != 1 || d->pad != 1) return LRD_ERR_UNSUPPORTED;
+    if (d->k < 1 || d->stride < 1 || d->pad < 0) return LRD_ERR_INVALID_ARG;
+    if (d->k > 7 || d->k % 2 == 0 || d->stride > 2 || d->pad != (d->k - 1) / 2) return LRD_ERR_UNSUPPORTED;
     if (d->H > 32767 || d->W > 32767) return LRD_ERR_UNSUPPORTED;
     return LRD_OK;
 }
@@ -98,7 +109,7 @@ size_t tucker2_workspace_bytes(const lrd_tucker2_desc_t* d, lrd_tucker_freeze_t 
         const lrd_tucker2_desc_t q = padded_desc(*d);
         return repack_layout(t, tucker2_workspace_bytes(&q, freeze, is_bwd)).total;
     }
-    return act_bytes(t, t.r1) + act_bytes(t, t.r2) + (is_bwd ? split_bytes(t) : 0);
+    return act_bytes(t, t.P, t.r1) + act_bytes(t, t.Po, t.r2) + (is_bwd ? split_bytes(t) : 0);
 }
 
 lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void* A, const void* G, const void* Bm,
@@ -119,19 +130,20 @@ lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void*
         LRD_TRY(tucker2_fwd(&q, X, w + o.A, w + o.G, w + o.Bm, bias, Y, Z1_save ? w + o.Z1 : nullptr, Z2_save ? w + o.Z2 : nullptr, freeze,
                             w, inner, path, s));
         if (Z1_save) LRD_TRY(copy2d_bf16(Z1_save, t.r1, w + o.Z1, q.r1, t.P, q.r1, t.r1, s));
-        if (Z2_save) LRD_TRY(copy2d_bf16(Z2_save, t.r2, w + o.Z2, q.r2, t.P, q.r2, t.r2, s));
+        if (Z2_save) LRD_TRY(copy2d_bf16(Z2_save, t.r2, w + o.Z2, q.r2, t.Po, q.r2, t.r2, s));
         return LRD_OK;
     }
     void* Z1 = Z1_save ? Z1_save : ws;
-    void* Z2 = Z2_save ? Z2_save : (void*)((uint8_t*)ws + act_bytes(t, t.r1));
+    void* Z2 = Z2_save ? Z2_save : (void*)((uint8_t*)ws + act_bytes(t, t.P, t.r1));
     LRD_TRY(run_gemm(make_gemm(t.P, t.r1, t.C, X, t.C, false, A, t.r1, true, Z1, t.r1, nullptr, t.dt), path, false, nullptr, 0, s));
     // core + last 1x1 in one launch where the shape allows: Z2 then stays on chip unless the caller saves it
-    if ((path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+    if (t.plain && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
         tc_conv_chain_eligible(false, t.B, t.H, t.W, t.r1, t.r2, t.S, t.dt, Z1, G, Bm, Y, Z2_save) &&
         (!bias || ((uintptr_t)bias % 2) == 0))
         return tc_conv3x3_chain(false, Z1, G, Bm, bias, Y, Z2_save, t.B, t.H, t.W, t.r1, t.r2, t.S, s);
-    LRD_TRY(conv3x3_fwd(Z1, G, Z2, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
-    return run_gemm(make_gemm(t.P, t.S, t.r2, Z2, t.r2, false, Bm, t.r2, false, Y, t.S, bias, t.dt), path, false, nullptr, 0, s);
+    if (t.plain) LRD_TRY(conv3x3_fwd(Z1, G, Z2, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    else LRD_TRY(simt_conv_fwd(Z1, G, Z2, t.B, t.g, t.r1, t.r2, t.dt, s));
+    return run_gemm(make_gemm(t.Po, t.S, t.r2, Z2, t.r2, false, Bm, t.r2, false, Y, t.S, bias, t.dt), path, false, nullptr, 0, s);
 }
 
 lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void* X, const void* A, const void* G,
@@ -146,7 +158,7 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
         LRD_TRY(zero_fill(dB, t.S, t.r2, t.r2, t.dt, s));
         LRD_TRY(zero_fill(dbias, 1, t.S, t.S, t.dt, s));
     }
-    if (!core || t.P == 0) LRD_TRY(zero_fill(dG, t.r2, 9 * t.r1, 9 * t.r1, t.dt, s));
+    if (!core || t.P == 0) LRD_TRY(zero_fill(dG, t.r2, t.taps * t.r1, t.taps * t.r1, t.dt, s));
     if (t.P == 0) return LRD_OK;
     if (needs_repack(t) && path != LRD_PATH_GENERAL) {
         const lrd_tucker2_desc_t q = padded_desc(*d);
@@ -158,7 +170,7 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
         LRD_TRY(zero_fill(w + o.G + (size_t)t.r2 * 9 * q.r1 * 2, (q.r2 - t.r2) * 9, q.r1, q.r1, LRD_BF16, s));
         LRD_TRY(copy2d_bf16(w + o.Bm, q.r2, Bm, t.r2, t.S, t.r2, q.r2, s));
         if (core) LRD_TRY(copy2d_bf16(w + o.Z1, q.r1, Z1_save, t.r1, t.P, t.r1, q.r1, s));
-        if (factors) LRD_TRY(copy2d_bf16(w + o.Z2, q.r2, Z2_save, t.r2, t.P, t.r2, q.r2, s));
+        if (factors) LRD_TRY(copy2d_bf16(w + o.Z2, q.r2, Z2_save, t.r2, t.Po, t.r2, q.r2, s));
         // the frozen group's buffers were zero-filled above; the padded call gets none for them
         LRD_TRY(tucker2_bwd(&q, dY, X, w + o.A, w + o.G, w + o.Bm, core ? w + o.Z1 : nullptr, factors ? w + o.Z2 : nullptr, dX,
                             factors ? w + o.dA : nullptr, core ? w + o.dG : nullptr, factors ? w + o.dB : nullptr, factors ? dbias : nullptr,
@@ -172,9 +184,9 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
     }
 
     void* dZ1 = ws;
-    void* dZ2 = (uint8_t*)ws + act_bytes(t, t.r1);
+    void* dZ2 = (uint8_t*)ws + act_bytes(t, t.P, t.r1);
     const Scratch reg = split_regions(t);
-    uint8_t* scratch0 = (uint8_t*)ws + act_bytes(t, t.r1) + act_bytes(t, t.r2);
+    uint8_t* scratch0 = (uint8_t*)ws + act_bytes(t, t.P, t.r1) + act_bytes(t, t.Po, t.r2);
     float* pB = (float*)scratch0;
     float* pA = (float*)(scratch0 + reg.dB);
     float* pF = (float*)(scratch0 + reg.dB + reg.dA);
@@ -193,33 +205,38 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
         if (!stream_after(sB, s, ss->fork)) return LRD_ERR_CUDA;
     }
     auto launch_dB = [&]() {
-        GemmArgs gb = make_gemm(t.S, t.r2, t.P, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt);
+        GemmArgs gb = make_gemm(t.S, t.r2, t.Po, dY, t.S, true, Z2_save, t.r2, true, dB, t.r2, nullptr, t.dt);
         bool db_done = false;
         if (dbias && path != LRD_PATH_GENERAL) {          // the bias gradient rides on the dB product (A = dY)
             gb.a_colsum = dbias;
             if (tc_gemm_colsum_ok(gb)) db_done = true; else gb.a_colsum = nullptr;
         }
         keep(run_gemm(gb, path, true, pB, reg.dB, sB));
-        if (dbias && !db_done) keep(colsum(dY, t.S, t.P, t.S, dbias, t.dt, pB, reg.dB, sB));
+        if (dbias && !db_done) keep(colsum(dY, t.S, t.Po, t.S, dbias, t.dt, pB, reg.dB, sB));
     };
     if (factors && sB != s) launch_dB();
 
-    keep(run_gemm(make_gemm(t.P, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
+    auto launch_filter = [&](cudaStream_t st_f) {
+        if (t.plain) keep(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, pF, reg.filter, st_f));
+        else keep(simt_conv_bwd_filter(dZ2, Z1_save, dG, t.B, t.g, t.r1, t.r2, t.dt, st_f));
+    };
+    keep(run_gemm(make_gemm(t.Po, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
     if (core && sF != s) {
         if (!stream_after(sF, s, ss->mid)) keep(LRD_ERR_CUDA);
-        else keep(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, pF, reg.filter, sF));
+        else launch_filter(sF);
     }
     // transposed core + first 1x1 (dX = dZ1 A^T) in one launch where the shape allows; dZ1 is written only for dA
-    const bool fuse_dx = dX && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+    const bool fuse_dx = dX && t.plain && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
                          tc_conv_chain_eligible(true, t.B, t.H, t.W, t.r1, t.r2, t.C, t.dt, dZ2, G, A, dX, factors ? dZ1 : nullptr);
     if (fuse_dx) keep(tc_conv3x3_chain(true, dZ2, G, A, nullptr, dX, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.r1, t.r2, t.C, s));
-    else if (dX || factors) keep(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    else if ((dX || factors) && t.plain) keep(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
+    else if (dX || factors) keep(simt_conv_bwd_data(dZ2, G, dZ1, t.B, t.g, t.r1, t.r2, t.dt, s));
     if (dX && !fuse_dx) keep(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
     if (factors) {
         if (sB == s) launch_dB();
         keep(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, pA, reg.dA, s));
     }
-    if (core && sF == s) keep(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, pF, reg.filter, s));
+    if (core && sF == s) launch_filter(s);
     // join even after a failed launch, so that a capture in progress is left whole
     if (sB != s && !stream_after(s, sB, ss->aux_done[0])) keep(LRD_ERR_CUDA);
     if (sF != s && !stream_after(s, sF, ss->aux_done[1])) keep(LRD_ERR_CUDA);
@@ -233,13 +250,13 @@ lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, in
                          int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
     if (path != LRD_PATH_GENERAL && tc_conv_eligible(B, H, W, ci, co, dt, in, G, out))
         return tc_conv3x3(false, in, G, out, B, H, W, ci, co, s);
-    return simt_conv3x3_fwd(in, G, out, B, H, W, ci, co, dt, s);
+    return simt_conv_fwd(in, G, out, B, conv_geom(H, W, 3, 1), ci, co, dt, s);
 }
 lrd_status_t conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W, int64_t ci,
                               int64_t co, lrd_dtype_t dt, int path, cudaStream_t s) {
     if (path != LRD_PATH_GENERAL && tc_conv_eligible(B, H, W, ci, co, dt, dout, G, din))
         return tc_conv3x3(true, dout, G, din, B, H, W, ci, co, s);
-    return simt_conv3x3_bwd_data(dout, G, din, B, H, W, ci, co, dt, s);
+    return simt_conv_bwd_data(dout, G, din, B, conv_geom(H, W, 3, 1), ci, co, dt, s);
 }
 lrd_status_t conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
                                 int64_t ci, int64_t co, lrd_dtype_t dt, int path, float* scratch, size_t scratch_bytes,
@@ -247,7 +264,7 @@ lrd_status_t conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int6
     if (path != LRD_PATH_GENERAL && tc_conv_eligible(B, H, W, ci, co, dt, dout, in, dG) &&
         scratch_bytes >= tc_conv_filter_scratch_bytes(B, H, W, ci, co))
         return tc_conv3x3_filter(dout, in, dG, B, H, W, ci, co, scratch, scratch_bytes, s);
-    return simt_conv3x3_bwd_filter(dout, in, dG, B, H, W, ci, co, dt, s);
+    return simt_conv_bwd_filter(dout, in, dG, B, conv_geom(H, W, 3, 1), ci, co, dt, s);
 }
 
 }  // namespace lrd

@@ -18,16 +18,26 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
 // after the other on the caller's stream.
 void tucker2_overlap(bool on);
 
-// General-path 3x3 core (stride 1, zero pad 1), NHWC, any channel counts.
-//   fwd:        out[p][o] = sum_{kh,kw,i} in[p + (kh-1, kw-1)][i] G[o][kh][kw][i]
-//   bwd_data:   din[p][i] = sum_{kh,kw,o} dout[p - (kh-1, kw-1)][o] G[o][kh][kw][i]
-//   bwd_filter: dG[o][kh][kw][i] = sum_p dout[p][o] in[p + (kh-1, kw-1)][i]
-lrd_status_t simt_conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
-                              int64_t co, lrd_dtype_t dt, cudaStream_t s);
-lrd_status_t simt_conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W,
-                                   int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s);
-lrd_status_t simt_conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
-                                     int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s);
+// Geometry of the k x k core: input H x W, output Ho x Wo = ((H - 1) / stride + 1) x ((W - 1) / stride + 1),
+// zero pad (k - 1) / 2.
+struct ConvGeom {
+    int H, W, Ho, Wo, k, stride, pad;
+};
+inline ConvGeom conv_geom(int64_t H, int64_t W, int64_t k, int64_t stride) {
+    return ConvGeom{(int)H, (int)W, (int)((H - 1) / stride + 1), (int)((W - 1) / stride + 1), (int)k, (int)stride, (int)((k - 1) / 2)};
+}
+
+// General-path k x k core, NHWC, any channel counts, any geometry above.  With p an output pixel and
+// p * stride + (kh, kw) - pad the input pixel its tap (kh, kw) looks at:
+//   fwd:        out[p][o] = sum_{kh,kw,i} in[p * stride + (kh, kw) - pad][i] G[o][kh][kw][i]
+//   bwd_data:   din[q][i] = sum over (p, kh, kw) with p * stride + (kh, kw) - pad = q, and o, of dout[p][o] G[o][kh][kw][i]
+//   bwd_filter: dG[o][kh][kw][i] = sum_p dout[p][o] in[p * stride + (kh, kw) - pad][i]
+lrd_status_t simt_conv_fwd(const void* in, const void* G, void* out, int64_t B, const ConvGeom& g, int64_t ci, int64_t co,
+                           lrd_dtype_t dt, cudaStream_t s);
+lrd_status_t simt_conv_bwd_data(const void* dout, const void* G, void* din, int64_t B, const ConvGeom& g, int64_t ci,
+                                int64_t co, lrd_dtype_t dt, cudaStream_t s);
+lrd_status_t simt_conv_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, const ConvGeom& g, int64_t ci,
+                                  int64_t co, lrd_dtype_t dt, cudaStream_t s);
 
 // Tensor-core 3x3 core (bf16, W <= 128, channel counts multiples of 8, 16-byte aligned bases).
 bool tc_conv_eligible(int64_t B, int64_t H, int64_t W, int64_t ci, int64_t co, lrd_dtype_t dt, const void* p0,
@@ -46,7 +56,7 @@ lrd_status_t tc_conv3x3_chain(bool dgrad, const void* img, const void* G, const 
 lrd_status_t tc_conv3x3_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W, int64_t ci,
                                int64_t co, float* scratch, size_t scratch_bytes, cudaStream_t s);
 
-// Path dispatch for the core (tensor-core kernel where the shape qualifies, else general).
+// Path dispatch for the 3x3, stride-1 core (tensor-core kernel where the shape qualifies, else general).
 lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
                          int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);
 lrd_status_t conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W, int64_t ci,

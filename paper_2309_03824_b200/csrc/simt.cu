@@ -56,36 +56,57 @@ template <typename T> struct PlainB {          // [N x K] (k contiguous) or [K x
     __device__ bool k_fastest() const { return !mn; }
     __device__ float operator()(int64_t k, int64_t n) const { return to_f32(mn ? p[k * ld + n] : p[n * ld + k]); }
 };
-// 3x3 taps of an NHWC image as the A operand: m = pixel, k = tap * C + channel; the tap offset is
-// sign * (kh - 1, kw - 1); pixels outside the image read as zero.
-template <typename T> struct ConvTapA {
-    const T* p; int H, W, C, sign;
+// k x k taps of an NHWC image as the A operand of the core's forward product: m = output pixel (b, ho, wo),
+// kidx = tap * C + channel; the tap (kh, kw) of output pixel (ho, wo) is input pixel (ho * stride + kh - pad,
+// wo * stride + kw - pad); pixels outside the image read as zero.
+template <typename T> struct ConvFwdA {
+    const T* p; ConvGeom g; int C;
     __device__ bool k_fastest() const { return true; }
-    __device__ float operator()(int64_t m, int64_t k) const {
-        const int t = (int)(k / C), c = (int)(k % C);
-        const int dh = sign * (t / 3 - 1), dw = sign * (t % 3 - 1);
-        const int w = (int)(m % W), h = (int)((m / W) % H);
-        if (h + dh < 0 || h + dh >= H || w + dw < 0 || w + dw >= W) return 0.f;
-        return to_f32(p[(m + (int64_t)dh * W + dw) * C + c]);
+    __device__ float operator()(int64_t m, int64_t kidx) const {
+        const int t = (int)(kidx / C), c = (int)(kidx % C);
+        const int wo = (int)(m % g.Wo), ho = (int)((m / g.Wo) % g.Ho);
+        const int64_t b = m / ((int64_t)g.Wo * g.Ho);
+        const int h = ho * g.stride + t / g.k - g.pad, w = wo * g.stride + t % g.k - g.pad;
+        if (h < 0 || h >= g.H || w < 0 || w >= g.W) return 0.f;
+        return to_f32(p[((b * g.H + h) * g.W + w) * C + c]);
     }
 };
-// One tap of an NHWC image as the B operand of the filter gradient: k = pixel, n = channel.
+// The same taps seen from the input side, as the A operand of the data gradient: m = input pixel (b, h, w),
+// kidx = tap * C + o; input pixel (h, w) met tap (kh, kw) of output pixel ((h + pad - kh) / stride,
+// (w + pad - kw) / stride) where both divisions are exact and the result lies inside the output.
+template <typename T> struct ConvBwdA {
+    const T* p; ConvGeom g; int C;
+    __device__ bool k_fastest() const { return true; }
+    __device__ float operator()(int64_t m, int64_t kidx) const {
+        const int t = (int)(kidx / C), c = (int)(kidx % C);
+        const int w = (int)(m % g.W), h = (int)((m / g.W) % g.H);
+        const int64_t b = m / ((int64_t)g.W * g.H);
+        const int hs = h + g.pad - t / g.k, ws = w + g.pad - t % g.k;
+        if (hs < 0 || ws < 0 || hs % g.stride || ws % g.stride) return 0.f;
+        const int ho = hs / g.stride, wo = ws / g.stride;
+        if (ho >= g.Ho || wo >= g.Wo) return 0.f;
+        return to_f32(p[((b * g.Ho + ho) * g.Wo + wo) * C + c]);
+    }
+};
+// One tap of an NHWC image as the B operand of the filter gradient: kidx = output pixel, n = channel.
 template <typename T> struct ConvTapB {
-    const T* p; int H, W, C, dh, dw;
+    const T* p; ConvGeom g; int C, kh, kw;
     __device__ bool k_fastest() const { return false; }
-    __device__ float operator()(int64_t k, int64_t n) const {
-        const int w = (int)(k % W), h = (int)((k / W) % H);
-        if (h + dh < 0 || h + dh >= H || w + dw < 0 || w + dw >= W) return 0.f;
-        return to_f32(p[(k + (int64_t)dh * W + dw) * C + n]);
+    __device__ float operator()(int64_t kidx, int64_t n) const {
+        const int wo = (int)(kidx % g.Wo), ho = (int)((kidx / g.Wo) % g.Ho);
+        const int64_t b = kidx / ((int64_t)g.Wo * g.Ho);
+        const int h = ho * g.stride + kh - g.pad, w = wo * g.stride + kw - g.pad;
+        if (h < 0 || h >= g.H || w < 0 || w >= g.W) return 0.f;
+        return to_f32(p[((b * g.H + h) * g.W + w) * C + n]);
     }
 };
-// The core G[o][tap][i] as the B operand of the data gradient: k = tap * Co + o, n = i.
+// The core G[o][tap][i] as the B operand of the data gradient: kidx = tap * Co + o, n = i.
 template <typename T> struct CoreTransposedB {
-    const T* p; int Ci, Co;
+    const T* p; int Ci, Co, taps;
     __device__ bool k_fastest() const { return false; }
-    __device__ float operator()(int64_t k, int64_t n) const {
-        const int64_t t = k / Co, o = k % Co;
-        return to_f32(p[(o * 9 + t) * Ci + n]);
+    __device__ float operator()(int64_t kidx, int64_t n) const {
+        const int64_t t = kidx / Co, o = kidx % Co;
+        return to_f32(p[(o * taps + t) * Ci + n]);
     }
 };
 
@@ -233,35 +254,43 @@ lrd_status_t simt_gemm_t(const GemmArgs& g, cudaStream_t stream) {
 }
 
 template <typename T>
-lrd_status_t conv_fwd_t(const void* in, const void* G, void* out, int64_t P, int H, int W, int ci, int co, int sign,
-                        bool transposed_core, cudaStream_t stream) {
-    // forward:  M = pixels, N = co, K = 9 ci, B = G as [co x 9 ci] (k contiguous)
-    // data grad: M = pixels, N = ci, K = 9 co, B = G regrouped as (tap, o) x i
-    const int64_t N = transposed_core ? ci : co, K = 9 * (int64_t)(transposed_core ? co : ci);
-    dim3 grid((unsigned)((N + TN - 1) / TN), (unsigned)((P + TM - 1) / TM));
-    ConvTapA<T> la{(const T*)in, H, W, transposed_core ? co : ci, sign};
-    if (transposed_core) {
-        CoreTransposedB<T> lb{(const T*)G, ci, co};
-        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, N, K, la, lb, (T*)out, N, (const T*)nullptr);
-    } else {
-        PlainB<T> lb{(const T*)G, 9 * (int64_t)ci, 0};
-        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, N, K, la, lb, (T*)out, N, (const T*)nullptr);
-    }
+lrd_status_t conv_fwd_t(const void* in, const void* G, void* out, int64_t B, const ConvGeom& g, int ci, int co, cudaStream_t stream) {
+    // M = output pixels, N = co, K = taps * ci, B = G as [co x taps * ci] (k contiguous)
+    const int64_t P = B * g.Ho * g.Wo, K = (int64_t)g.k * g.k * ci;
+    dim3 grid((unsigned)((co + TN - 1) / TN), (unsigned)((P + TM - 1) / TM));
+    ConvFwdA<T> la{(const T*)in, g, ci};
+    PlainB<T> lb{(const T*)G, K, 0};
+    simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, co, K, la, lb, (T*)out, co, (const T*)nullptr);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
 template <typename T>
-lrd_status_t conv_filter_t(const void* dout, const void* in, void* dG, int64_t P, int H, int W, int ci, int co,
+lrd_status_t conv_bwd_data_t(const void* dout, const void* G, void* din, int64_t B, const ConvGeom& g, int ci, int co,
+                             cudaStream_t stream) {
+    // M = input pixels, N = ci, K = taps * co, B = G regrouped as (tap, o) x i
+    const int64_t P = B * g.H * g.W, K = (int64_t)g.k * g.k * co;
+    dim3 grid((unsigned)((ci + TN - 1) / TN), (unsigned)((P + TM - 1) / TM));
+    ConvBwdA<T> la{(const T*)dout, g, co};
+    CoreTransposedB<T> lb{(const T*)G, ci, co, g.k * g.k};
+    simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(P, ci, K, la, lb, (T*)din, ci, (const T*)nullptr);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
+}
+
+template <typename T>
+lrd_status_t conv_filter_t(const void* dout, const void* in, void* dG, int64_t B, const ConvGeom& g, int ci, int co,
                            cudaStream_t stream) {
+    const int taps = g.k * g.k;
+    const int64_t P = B * g.Ho * g.Wo;
     dim3 grid((unsigned)((ci + TN - 1) / TN), (unsigned)((co + TM - 1) / TM));
-    for (int t = 0; t < 9; ++t) {      // one product per tap: M = co, N = ci, K = pixels (single block owns all of K)
+    for (int t = 0; t < taps; ++t) {   // one product per tap: M = co, N = ci, K = output pixels (single block owns all of K)
         PlainA<T> la{(const T*)dout, co, 1};
-        ConvTapB<T> lb{(const T*)in, H, W, ci, t / 3 - 1, t % 3 - 1};
-        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(co, ci, P, la, lb, (T*)dG + (int64_t)t * ci, 9 * (int64_t)ci,
+        ConvTapB<T> lb{(const T*)in, g, ci, t / g.k, t % g.k};
+        simt_gemm_kernel<T><<<grid, NT, 0, stream>>>(co, ci, P, la, lb, (T*)dG + (int64_t)t * ci, (int64_t)taps * ci,
                                                      (const T*)nullptr);
     }
-    count_launch(9);
+    count_launch(taps);
     return cudaGetLastError() == cudaSuccess ? LRD_OK : LRD_ERR_CUDA;
 }
 
@@ -272,20 +301,20 @@ lrd_status_t simt_gemm(const GemmArgs& g, cudaStream_t stream) {
     return g.dtype == LRD_F32 ? simt_gemm_t<float>(g, stream) : simt_gemm_t<__nv_bfloat16>(g, stream);
 }
 
-lrd_status_t simt_conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
-                              int64_t co, lrd_dtype_t dt, cudaStream_t s) {
-    return dt == LRD_F32 ? conv_fwd_t<float>(in, G, out, B * H * W, (int)H, (int)W, (int)ci, (int)co, 1, false, s)
-                         : conv_fwd_t<__nv_bfloat16>(in, G, out, B * H * W, (int)H, (int)W, (int)ci, (int)co, 1, false, s);
+lrd_status_t simt_conv_fwd(const void* in, const void* G, void* out, int64_t B, const ConvGeom& g, int64_t ci, int64_t co,
+                           lrd_dtype_t dt, cudaStream_t s) {
+    return dt == LRD_F32 ? conv_fwd_t<float>(in, G, out, B, g, (int)ci, (int)co, s)
+                         : conv_fwd_t<__nv_bfloat16>(in, G, out, B, g, (int)ci, (int)co, s);
 }
-lrd_status_t simt_conv3x3_bwd_data(const void* dout, const void* G, void* din, int64_t B, int64_t H, int64_t W,
-                                   int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s) {
-    return dt == LRD_F32 ? conv_fwd_t<float>(dout, G, din, B * H * W, (int)H, (int)W, (int)ci, (int)co, -1, true, s)
-                         : conv_fwd_t<__nv_bfloat16>(dout, G, din, B * H * W, (int)H, (int)W, (int)ci, (int)co, -1, true, s);
+lrd_status_t simt_conv_bwd_data(const void* dout, const void* G, void* din, int64_t B, const ConvGeom& g, int64_t ci,
+                                int64_t co, lrd_dtype_t dt, cudaStream_t s) {
+    return dt == LRD_F32 ? conv_bwd_data_t<float>(dout, G, din, B, g, (int)ci, (int)co, s)
+                         : conv_bwd_data_t<__nv_bfloat16>(dout, G, din, B, g, (int)ci, (int)co, s);
 }
-lrd_status_t simt_conv3x3_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W,
-                                     int64_t ci, int64_t co, lrd_dtype_t dt, cudaStream_t s) {
-    return dt == LRD_F32 ? conv_filter_t<float>(dout, in, dG, B * H * W, (int)H, (int)W, (int)ci, (int)co, s)
-                         : conv_filter_t<__nv_bfloat16>(dout, in, dG, B * H * W, (int)H, (int)W, (int)ci, (int)co, s);
+lrd_status_t simt_conv_bwd_filter(const void* dout, const void* in, void* dG, int64_t B, const ConvGeom& g, int64_t ci,
+                                  int64_t co, lrd_dtype_t dt, cudaStream_t s) {
+    return dt == LRD_F32 ? conv_filter_t<float>(dout, in, dG, B, g, (int)ci, (int)co, s)
+                         : conv_filter_t<__nv_bfloat16>(dout, in, dG, B, g, (int)ci, (int)co, s);
 }
 
 int colsum_splits(int64_t M) {

@@ -113,15 +113,17 @@ def tucker_case(B, H, W, C, S, r1, r2, k, dtype, seed_base, decompose, with_bias
     return case
 
 
-def random_tucker_case(B, H, W, C, S, r1, r2, k, dtype, seed_base, with_bias=True):
-    """Tucker-2 layer with directly drawn factors (no decomposition), unit-scale activations."""
+def random_tucker_case(B, H, W, C, S, r1, r2, k, dtype, seed_base, with_bias=True, stride=1):
+    """Tucker-2 layer with directly drawn factors (no decomposition), unit-scale activations.  The output (and dY)
+    has (H - 1) // stride + 1 rows and (W - 1) // stride + 1 columns of pixels."""
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
     case = {
         "X": round_to(normal(seed_base + 1, (B, H, W, C)), dtype),
         "A": round_to(normal(seed_base + 4, (C, r1), C ** -0.5), dtype),
         "G": round_to(normal(seed_base + 5, (r2, k, k, r1), (k * k * r1) ** -0.5), dtype),
         "Bm": round_to(normal(seed_base + 6, (S, r2), r2 ** -0.5), dtype),
-        "dY": round_to(normal(seed_base + 3, (B, H, W, S)), dtype),
-        "B": B, "H": H, "W": W, "C": C, "S": S, "r1": r1, "r2": r2, "k": k, "dtype": dtype,
+        "dY": round_to(normal(seed_base + 3, (B, Ho, Wo, S)), dtype),
+        "B": B, "H": H, "W": W, "C": C, "S": S, "r1": r1, "r2": r2, "k": k, "stride": stride, "dtype": dtype,
     }
     case["b"] = round_to(normal(seed_base + 2, (S,), BIAS_STD), dtype) if with_bias else None
     return case

@@ -1,4 +1,4 @@
-"""GPU parity of the Tucker-2 decomposed 3x3 convolution against the CPU oracle, through the C ABI."""
+"""GPU parity of the Tucker-2 decomposed convolution against the CPU oracle, through the C ABI."""
 import numpy as np
 import pytest
 import torch
@@ -18,19 +18,21 @@ def run_tucker(case, freeze, path=b.LRD_PATH_AUTO, want_dx=True):
     dt = case["dtype"]
     code, tdt = DT[dt]
     B, H, W, C, S, r1, r2 = (case[k] for k in ("B", "H", "W", "C", "S", "r1", "r2"))
-    desc = b.tucker2_desc(B, H, W, C, S, r1, r2, code)
+    k, stride = case.get("k", 3), case.get("stride", 1)
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    desc = b.tucker2_desc(B, H, W, C, S, r1, r2, code, k=k, stride=stride, pad=(k - 1) // 2)
     X, A, G, Bm, bias, dY = (dev(case[k], dt) for k in ("X", "A", "G", "Bm", "b", "dY"))
     ws = workspace(max(b.lrd_tucker2_workspace_bytes(desc, freeze, 0), b.lrd_tucker2_workspace_bytes(desc, freeze, 1)))
     b.lrd_set_path(path)
     try:
-        Y = torch.empty(B, H, W, S, dtype=tdt, device="cuda")
+        Y = torch.empty(B, Ho, Wo, S, dtype=tdt, device="cuda")
         Z1 = None if freeze == b.LRD_TK_FREEZE_CORE else torch.empty(B, H, W, r1, dtype=tdt, device="cuda")
-        Z2 = None if freeze == b.LRD_TK_FREEZE_FACTORS else torch.empty(B, H, W, r2, dtype=tdt, device="cuda")
+        Z2 = None if freeze == b.LRD_TK_FREEZE_FACTORS else torch.empty(B, Ho, Wo, r2, dtype=tdt, device="cuda")
         b.lrd_tucker2_fwd(desc, X, A, G, Bm, bias, Y, Z1, Z2, freeze, ws)
         nan = float("nan")
         dX = torch.full((B, H, W, C), nan, dtype=tdt, device="cuda") if want_dx else None
         dA = torch.full((C, r1), nan, dtype=tdt, device="cuda")
-        dG = torch.full((r2, 3, 3, r1), nan, dtype=tdt, device="cuda")
+        dG = torch.full((r2, k, k, r1), nan, dtype=tdt, device="cuda")
         dB = torch.full((S, r2), nan, dtype=tdt, device="cuda")
         db = torch.full((S,), nan, dtype=tdt, device="cuda")
         b.lrd_tucker2_bwd(desc, dY, None if freeze == b.LRD_TK_FREEZE_FACTORS else X, A, G, Bm, Z1, Z2, dX, dA, dG, dB, db,
@@ -44,8 +46,9 @@ def run_tucker(case, freeze, path=b.LRD_PATH_AUTO, want_dx=True):
 
 def check_tucker(case, freeze, path=b.LRD_PATH_AUTO, tol=None):
     got = run_tucker(case, freeze, path)
-    Z1, Z2, Y = o.tucker2_fwd(case["X"], case["A"], case["G"], case["Bm"], case["b"])
-    ref = o.tucker2_bwd(case["dY"], case["X"], case["A"], case["G"], case["Bm"], Z1, Z2, freeze)
+    stride = case.get("stride", 1)
+    Z1, Z2, Y = o.tucker2_fwd(case["X"], case["A"], case["G"], case["Bm"], case["b"], stride)
+    ref = o.tucker2_bwd(case["dY"], case["X"], case["A"], case["G"], case["Bm"], Z1, Z2, freeze, stride)
     ref.update({"Y": Y, "Z1": Z1, "Z2": Z2})
     tol = TOL[case["dtype"]] if tol is None else tol
     errs = {k: rel_err(v, ref[k]) for k, v in got.items() if v is not None}
@@ -63,6 +66,30 @@ def check_tucker(case, freeze, path=b.LRD_PATH_AUTO, tol=None):
 def test_general_path_small_geometries(dtype, geom, freeze):
     B, H, W, C, S, r1, r2 = geom
     check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, dtype, 400 + H), freeze, path=b.LRD_PATH_GENERAL)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("geom", [(2, 8, 8, 16, 24, 8, 16, 3, 2), (2, 7, 9, 12, 10, 5, 6, 3, 2), (1, 1, 1, 4, 4, 2, 3, 3, 2), (2, 6, 5, 16, 16, 8, 8, 5, 1),
+                                  (2, 9, 7, 12, 20, 6, 7, 5, 2), (2, 5, 6, 24, 16, 8, 16, 1, 1), (3, 7, 7, 16, 24, 16, 8, 1, 2),
+                                  (1, 8, 9, 8, 8, 4, 4, 7, 1), (4, 14, 14, 64, 128, 32, 40, 3, 2)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_strided_and_wider_cores(dtype, geom, freeze):
+    """k x k cores with k = 1, 3, 5, 7 and stride 1 or 2 (the downsampling blocks of a residual network carry their
+    stride on the 3 x 3 convolution): the 1 x 1 products run wherever their shapes allow, the core on the general
+    kernels; Z2, Y and dY live on the strided output grid."""
+    B, H, W, C, S, r1, r2, k, stride = geom
+    check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, k, dtype, 470 + H + k + stride, stride=stride), freeze)
+
+
+def test_geometries_outside_the_supported_set_are_refused():
+    t = torch.zeros(1 << 12, dtype=torch.float32, device="cuda")
+    ws = workspace(1 << 16)
+    for k, stride, pad, want in ((4, 1, 1, b.LRD_ERR_UNSUPPORTED), (9, 1, 4, b.LRD_ERR_UNSUPPORTED), (3, 3, 1, b.LRD_ERR_UNSUPPORTED),
+                                 (3, 1, 0, b.LRD_ERR_UNSUPPORTED), (5, 1, 1, b.LRD_ERR_UNSUPPORTED), (0, 1, 0, b.LRD_ERR_INVALID_ARG),
+                                 (3, 0, 1, b.LRD_ERR_INVALID_ARG)):
+        d = b.tucker2_desc(1, 4, 4, 4, 4, 2, 2, b.LRD_F32, k=k, stride=stride, pad=pad)
+        assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, t, t, 0, ws, check=False) == want, (k, stride, pad)
+        assert b.lrd_tucker2_workspace_bytes(d, 0, 0) == 0
 
 
 @pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 9, 11, 128, 136, 96, 104), (5, 14, 14, 256, 256, 96, 96),
@@ -152,7 +179,7 @@ def test_argument_checks():
     assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, t, t, b.LRD_TK_FREEZE_CORE, ws, check=False) == b.LRD_ERR_INVALID_ARG
     assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, None, t, b.LRD_TK_FREEZE_NONE, ws, check=False) == b.LRD_ERR_INVALID_ARG
     assert b.lrd_tucker2_fwd(d, t, t, t, t, None, t, t, t, b.LRD_TK_FREEZE_FACTORS, ws, check=False) == b.LRD_ERR_INVALID_ARG
-    bad = b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, code, k=5, pad=2)
+    bad = b.tucker2_desc(1, 4, 4, 8, 8, 4, 4, code, k=4, pad=1)
     assert b.lrd_tucker2_fwd(bad, t, t, t, t, None, t, t, t, 0, ws, check=False) == b.LRD_ERR_UNSUPPORTED
     bad = b.tucker2_desc(1, 4, 4, 8, 8, 9, 4, code)
     assert b.lrd_tucker2_fwd(bad, t, t, t, t, None, t, t, t, 0, ws, check=False) == b.LRD_ERR_BAD_RANK

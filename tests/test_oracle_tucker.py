@@ -146,3 +146,81 @@ def test_tucker_backward_finite_differences_and_masks():
     assert np.array_equal(ff["dG"], gr["dG"]) and np.array_equal(ff["dX"], gr["dX"])
     for n in ("dA", "dB", "db", "dX"):
         assert np.array_equal(fc[n], gr[n])
+
+
+def conv_brute_strided(X, Wk, pad, stride):
+    """The definition again, with a stride: output pixel (ho, wo) looks at input rows ho * stride + kh - pad."""
+    B, H, W, Ci = X.shape
+    Co, k, _, _ = Wk.shape
+    Ho, Wo = (H + 2 * pad - k) // stride + 1, (W + 2 * pad - k) // stride + 1
+    Y = np.zeros((B, Ho, Wo, Co))
+    for b in range(B):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                for co in range(Co):
+                    acc = 0.0
+                    for kh in range(k):
+                        for kw in range(k):
+                            hh, ww = ho * stride + kh - pad, wo * stride + kw - pad
+                            if 0 <= hh < H and 0 <= ww < W:
+                                for ci in range(Ci):
+                                    acc += X[b, hh, ww, ci] * Wk[co, kh, kw, ci]
+                    Y[b, ho, wo, co] = acc
+    return Y
+
+
+@pytest.mark.parametrize("k,stride,hw", [(3, 2, (5, 6)), (3, 2, (4, 4)), (5, 1, (5, 4)), (5, 2, (7, 5)), (1, 2, (5, 5)), (7, 1, (4, 6))])
+def test_strided_and_wider_convolutions(k, stride, hw):
+    """Forward against brute force and against the stride-1 result sampled every `stride` pixels; the gradients
+    as adjoints of the forward map and against finite differences."""
+    g = rng(40 + k + stride)
+    H, W = hw
+    pad = (k - 1) // 2
+    X, Wk = g.standard_normal((2, H, W, 3)), g.standard_normal((4, k, k, 3))
+    Y = o.conv2d_nhwc_fwd(X, Wk, pad, stride)
+    assert Y.shape == (2, (H - 1) // stride + 1, (W - 1) // stride + 1, 4)
+    assert np.abs(Y - conv_brute_strided(X, Wk, pad, stride)).max() <= 1e-13
+    assert np.abs(Y - o.conv2d_nhwc_fwd(X, Wk, pad, 1)[:, ::stride, ::stride, :]).max() <= 1e-13
+    dY = g.standard_normal(Y.shape)
+    dX = o.conv2d_nhwc_bwd_data(dY, Wk, pad, (H, W), stride)
+    dW = o.conv2d_nhwc_bwd_filter(dY, X, k, pad, stride)
+    assert dX.shape == X.shape and dW.shape == Wk.shape
+    L = float(np.sum(Y * dY))
+    assert abs(np.sum(dX * X) - L) <= 1e-11 * abs(L) + 1e-12
+    assert abs(np.sum(dW * Wk) - L) <= 1e-11 * abs(L) + 1e-12
+    eps = 1e-6
+    for which, (arr, grad) in enumerate(((X, dX), (Wk, dW))):
+        for _ in range(6):
+            idx = tuple(int(g.integers(0, n)) for n in arr.shape)
+            hi, lo = arr.copy(), arr.copy()
+            hi[idx] += eps
+            lo[idx] -= eps
+            f = (lambda a: np.sum(o.conv2d_nhwc_fwd(a, Wk, pad, stride) * dY)) if which == 0 else \
+                (lambda a: np.sum(o.conv2d_nhwc_fwd(X, a, pad, stride) * dY))
+            assert abs((f(hi) - f(lo)) / (2 * eps) - grad[idx]) <= 1e-7 * max(1.0, abs(grad[idx]))
+
+
+@pytest.mark.parametrize("k,stride", [(3, 2), (5, 1), (1, 1)])
+def test_tucker2_layer_with_stride_equals_the_dense_convolution_and_its_gradients(k, stride):
+    """Forward = dense convolution with the reconstructed kernel at the same stride; every gradient against finite
+    differences of the forward map."""
+    g = rng(70 + k + stride)
+    B, H, W, C, S, r1, r2 = 2, 5, 4, 4, 5, 3, 2
+    X, A, G, Bm = g.standard_normal((B, H, W, C)), g.standard_normal((C, r1)), g.standard_normal((r2, k, k, r1)), g.standard_normal((S, r2))
+    bias = g.standard_normal(S)
+    Z1, Z2, Y = o.tucker2_fwd(X, A, G, Bm, bias, stride)
+    Wd = o.tucker2_reconstruct(A, G, Bm)                      # [S][C][k][k]
+    ref = o.conv2d_nhwc_fwd(X, np.transpose(Wd, (0, 2, 3, 1)), (k - 1) // 2, stride) + bias
+    assert np.abs(Y - ref).max() <= 1e-12
+    dY = g.standard_normal(Y.shape)
+    gr = o.tucker2_bwd(dY, X, A, G, Bm, Z1, Z2, o.TK_FREEZE_NONE, stride)
+    vals = [X, A, G, Bm, bias]
+    eps = 1e-6
+    for pos, name in ((0, "dX"), (1, "dA"), (2, "dG"), (3, "dB"), (4, "db")):
+        for _ in range(4):
+            idx = tuple(int(g.integers(0, n)) for n in vals[pos].shape)
+            hi, lo = [v.copy() for v in vals], [v.copy() for v in vals]
+            hi[pos][idx] += eps
+            lo[pos][idx] -= eps
+            fd = (np.sum(o.tucker2_fwd(*hi, stride)[2] * dY) - np.sum(o.tucker2_fwd(*lo, stride)[2] * dY)) / (2 * eps)
+            assert abs(fd - gr[name][idx]) <= 1e-7 * max(1.0, abs(gr[name][idx])), name

@@ -28,9 +28,9 @@ namespace {
 using namespace ptx;
 
 constexpr int kThreads = 192;
-constexpr int kStages = 4;
+constexpr int kStages = 6;                           // what a block streams is its stages in flight over a stage's turn-around
 constexpr uint32_t kTile = 128 * 128;               // one operand tile slot: 128 rows x 64 channels of bf16
-constexpr uint32_t kStageBytes = 3 * kTile;          // A slot + two 64-wide B slots (N = 128)
+constexpr uint32_t kStageBytes = 2 * kTile;          // A slot + B slot (N = 128: one K-major tile or two 64-wide MN-major boxes)
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024;
 
 struct ConvParams {

@@ -44,15 +44,26 @@ class Timing(float):
 
 
 def _time(fn, iters, repeats=3):
-    for _ in range(3):
+    """Seconds per call of fn: `iters` calls captured into one CUDA graph (what is timed is then the GPU's time, not
+    the host's launch path, which at these sizes is the longer of the two and the noisier), replayed `repeats` times
+    after a warm-up replay; the fastest replay counts, the spread of the replays is kept beside it."""
+    for _ in range(3):                      # eager first: the library creates its side streams outside a capture
         fn()
     torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(iters):
+                fn()
+    torch.cuda.synchronize()
+    graph.replay()
     out = []
     for _ in range(repeats):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
         e0.record()
-        for _ in range(iters):
-            fn()
+        graph.replay()
         e1.record()
         torch.cuda.synchronize()
         out.append(e0.elapsed_time(e1) * 1e-3 / iters)

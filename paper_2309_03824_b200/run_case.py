@@ -5,8 +5,9 @@ profilers and quick timing.
 
 --r 0 runs the undecomposed layer (lrd_dense_fwd / lrd_dense_bwd) instead.  --tucker B,H,W,C,S,r1,r2 runs a Tucker-2
 decomposed 3 x 3 convolution (lrd_tucker2_fwd / lrd_tucker2_bwd; --freeze none | factors | core).  --dtype f32 runs
-the linear layer in fp32 (the general fp32-FMA kernels).  --packed-odd stores the factors packed at the given rank
-even when it is not a multiple of 8 (the repacking path).
+the linear layer in fp32 (the general fp32-FMA kernels).  Factors are stored packed, so a rank that is not a multiple
+of 8 (--r 250) takes the repacking path.  --accumulate runs the backward pass through lrd_linear_bwd_accumulate (the
+gradients are added to what the buffers hold).
 """
 from __future__ import annotations
 
@@ -58,6 +59,7 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--what", default="both", choices=["fwd", "bwd", "both"])
     ap.add_argument("--path", default="auto", choices=["auto", "general", "unfused", "fused"])
+    ap.add_argument("--accumulate", action="store_true")
     a = ap.parse_args()
     b.lrd_set_path({"auto": 0, "general": 1, "unfused": 2, "fused": 3}[a.path])
     if a.tucker:
@@ -80,9 +82,12 @@ def main():
         sets.append(dict(X=torch.from_numpy(case["X"]).to("cuda", bf), dY=torch.from_numpy(case["dY"]).to("cuda", bf),
                          Y=torch.empty(a.M, a.N, dtype=bf, device="cuda"), Z=torch.empty(a.M, max(a.r, 8), dtype=bf, device="cuda"),
                          dX=torch.empty(a.M, a.K, dtype=bf, device="cuda")))
-    dU = torch.empty(a.N, a.r, dtype=bf, device="cuda")
-    dV = torch.empty(a.K, a.r, dtype=bf, device="cuda")
-    db = torch.empty(a.N, dtype=bf, device="cuda")
+    dU = torch.zeros(a.N, a.r, dtype=bf, device="cuda")
+    dV = torch.zeros(a.K, a.r, dtype=bf, device="cuda")
+    db = torch.zeros(a.N, dtype=bf, device="cuda")
+    if a.accumulate and not dense:
+        ws = torch.empty(max(b.lrd_linear_workspace_bytes(desc, freeze, 2), 256), dtype=torch.uint8, device="cuda")
+    bwd = b.lrd_linear_bwd_accumulate if a.accumulate else b.lrd_linear_bwd
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for phase in ("warm", "timed"):
         torch.cuda.synchronize()
@@ -98,9 +103,9 @@ def main():
             if a.what in ("fwd", "both"):
                 b.lrd_linear_fwd(desc, s["X"], V, U, bias, s["Y"], None if freeze == 1 else s["Z"], freeze, ws)
             if a.what in ("bwd", "both"):
-                b.lrd_linear_bwd(desc, s["dY"], None if freeze == 2 else s["X"], V, U, None if freeze == 1 else s["Z"],
-                                 s["dX"], None if freeze == 1 else dU, None if freeze == 2 else dV,
-                                 None if freeze == 1 else db, freeze, ws)
+                bwd(desc, s["dY"], None if freeze == 2 else s["X"], V, U, None if freeze == 1 else s["Z"],
+                    s["dX"], None if freeze == 1 else dU, None if freeze == 2 else dV,
+                    None if freeze == 1 else db, freeze, ws)
         e1.record()
         torch.cuda.synchronize()
     st = b.lrd_check_device_status()

@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture of
 # the 768->3072, r=384 forward; summary in profiles/chain_kernel_ffn1_forward.md).  It is reported only while the
 # kernel's sources still have the digest the capture was taken with.
-NCU_TRAFFIC = {"digest": "6fcb75b6a4dd3427", "bytes_per_launch": 9319936, "l2_to_sm_bytes_per_launch": 129171456,
+NCU_TRAFFIC = {"digest": "43a48a7824f353d6", "bytes_per_launch": 9320192, "l2_to_sm_bytes_per_launch": 129171456,
                "note": "DRAM reads of the launch (X and the weights once); its 25 MB of output were still in the 126 MB L2 when "
                        "the counters stopped, so this is below the algorithmic bytes and says only that nothing is re-read from HBM"}
 KERNEL_SOURCES = ("paper_2309_03824_b200/csrc/chain.cu", "paper_2309_03824_b200/csrc/ptx.cuh")

@@ -304,7 +304,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
         fence_proxy_async_smem();
         tc_fence_before();
         cluster_wait();        // barrier 1: the peers' barriers exist
-        named_bar_sync(2, 128);
+        ok = named_bar_and(2, 128, ok);    // the four warps go on, or give up, together
         if (lead_warp) {
             if (ok && elect_one()) {
                 const uint32_t slice = t_base + (uint32_t)c * 256u * (uint32_t)p.RS;

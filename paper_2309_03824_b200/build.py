@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblrd_b200.so")
-SOURCES = ["lrd_api.cu", "simt.cu", "tma.cu", "tc_gemm.cu", "tc_gemm_persistent.cu", "chain.cu", "chain_pair.cu", "conv.cu", "conv_tc.cu", "streams.cu", "selftest.cu"]
+SOURCES = ["lrd_api.cu", "simt.cu", "tma.cu", "tc_gemm.cu", "tc_gemm_persistent.cu", "chain.cu", "chain_pair.cu", "conv.cu", "conv_tc.cu", "tucker_fused.cu", "streams.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-cudart", "static"]
 

@@ -133,6 +133,10 @@ lrd_status_t tucker2_fwd(const lrd_tucker2_desc_t* d, const void* X, const void*
         if (Z2_save) LRD_TRY(copy2d_bf16(Z2_save, t.r2, w + o.Z2, q.r2, t.Po, q.r2, t.r2, s));
         return LRD_OK;
     }
+    // the whole forward in one launch where the shape allows: Z1 and Z2 stay on chip unless the caller saves them
+    if (t.plain && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) && (!bias || ((uintptr_t)bias % 2) == 0) &&
+        tucker_fused_eligible(t.B, t.H, t.W, t.C, t.r1, t.r2, t.S, t.dt, X, A, G, Bm, Y, Z1_save, Z2_save))
+        return tucker_fused(false, X, A, G, Bm, bias, Y, Z1_save, Z2_save, t.B, t.H, t.W, t.C, t.r1, t.r2, t.S, s);
     void* Z1 = Z1_save ? Z1_save : ws;
     void* Z2 = Z2_save ? Z2_save : (void*)((uint8_t*)ws + act_bytes(t, t.P, t.r1));
     LRD_TRY(run_gemm(make_gemm(t.P, t.r1, t.C, X, t.C, false, A, t.r1, true, Z1, t.r1, nullptr, t.dt), path, false, nullptr, 0, s));
@@ -220,18 +224,30 @@ lrd_status_t tucker2_bwd(const lrd_tucker2_desc_t* d, const void* dY, const void
         if (t.plain) keep(conv3x3_bwd_filter(dZ2, Z1_save, dG, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, pF, reg.filter, st_f));
         else keep(simt_conv_bwd_filter(dZ2, Z1_save, dG, t.B, t.g, t.r1, t.r2, t.dt, st_f));
     };
-    keep(run_gemm(make_gemm(t.Po, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
+    // the whole data path (dZ2 = dY Bm, transposed core, dX = dZ1 A^T) in one launch where the shape allows; dZ2 is
+    // written only for the filter gradient, dZ1 only for dA.  (Giving the filter gradient a dZ2 product of its own
+    // beside the pass, so that it need not wait for it, was slower: 44.5 against 41.2 us per step with the core
+    // unfrozen -- the extra launch takes SMs from the pass.)
+    const bool one_launch = dX && t.plain && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+                            tucker_fused_eligible(t.B, t.H, t.W, t.S, t.r2, t.r1, t.C, t.dt, dY, Bm, G, A, dX, core ? dZ2 : nullptr,
+                                                  factors ? dZ1 : nullptr);
+    if (one_launch)
+        keep(tucker_fused(true, dY, Bm, G, A, nullptr, dX, core ? dZ2 : nullptr, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.S, t.r2,
+                          t.r1, t.C, s));
+    else
+        keep(run_gemm(make_gemm(t.Po, t.r2, t.S, dY, t.S, false, Bm, t.r2, true, dZ2, t.r2, nullptr, t.dt), path, false, nullptr, 0, s));
     if (core && sF != s) {
         if (!stream_after(sF, s, ss->mid)) keep(LRD_ERR_CUDA);
         else launch_filter(sF);
     }
     // transposed core + first 1x1 (dX = dZ1 A^T) in one launch where the shape allows; dZ1 is written only for dA
-    const bool fuse_dx = dX && t.plain && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
+    const bool fuse_dx = !one_launch && dX && t.plain && (path == LRD_PATH_AUTO || path == LRD_PATH_FUSED) &&
                          tc_conv_chain_eligible(true, t.B, t.H, t.W, t.r1, t.r2, t.C, t.dt, dZ2, G, A, dX, factors ? dZ1 : nullptr);
-    if (fuse_dx) keep(tc_conv3x3_chain(true, dZ2, G, A, nullptr, dX, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.r1, t.r2, t.C, s));
+    if (one_launch) {
+    } else if (fuse_dx) keep(tc_conv3x3_chain(true, dZ2, G, A, nullptr, dX, factors ? dZ1 : nullptr, t.B, t.H, t.W, t.r1, t.r2, t.C, s));
     else if ((dX || factors) && t.plain) keep(conv3x3_bwd_data(dZ2, G, dZ1, t.B, t.H, t.W, t.r1, t.r2, t.dt, path, s));
     else if (dX || factors) keep(simt_conv_bwd_data(dZ2, G, dZ1, t.B, t.g, t.r1, t.r2, t.dt, s));
-    if (dX && !fuse_dx) keep(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
+    if (dX && !fuse_dx && !one_launch) keep(run_gemm(make_gemm(t.P, t.C, t.r1, dZ1, t.r1, false, A, t.r1, false, dX, t.C, nullptr, t.dt), path, false, nullptr, 0, s));
     if (factors) {
         if (sB == s) launch_dB();
         keep(run_gemm(make_gemm(t.C, t.r1, t.P, X, t.C, true, dZ1, t.r1, true, dA, t.r1, nullptr, t.dt), path, true, pA, reg.dA, s));

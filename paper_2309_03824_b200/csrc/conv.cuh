@@ -56,6 +56,18 @@ lrd_status_t tc_conv3x3_chain(bool dgrad, const void* img, const void* G, const 
 lrd_status_t tc_conv3x3_filter(const void* dout, const void* in, void* dG, int64_t B, int64_t H, int64_t W, int64_t ci,
                                int64_t co, float* scratch, size_t scratch_bytes, cudaStream_t s);
 
+// A whole data pass of the layer in one launch (3 x 3 core, stride 1; ranks <= 128 and multiples of 16, at most 256 output
+// channels, images at most 40 pixels wide): forward (dgrad = false) out3 = conv(in P1, G) P3^T + bias3 with P1 = A [C x r1],
+// P3 = Bm [S x r2]; backward (dgrad = true) out3 = conv^T(in P1, G) P3^T with in = dY, P1 = Bm [S x r2], P3 = A [C x r1].
+// c_in = channels of `in`, nA = columns of P1, nB = channels after the core, n3 = rows of P3 = columns of out3.  save1
+// [pixels x nA] / save2 [pixels x nB] (nullable) receive the two intermediates where the caller needs them later.
+bool tucker_fused_eligible(int64_t B, int64_t H, int64_t W, int64_t c_in, int64_t nA, int64_t nB, int64_t n3, lrd_dtype_t dt,
+                           const void* in, const void* P1, const void* G, const void* P3, const void* out3, const void* save1,
+                           const void* save2);
+lrd_status_t tucker_fused(bool dgrad, const void* in, const void* P1, const void* G, const void* P3, const void* bias3, void* out3,
+                          void* save1, void* save2, int64_t B, int64_t H, int64_t W, int64_t c_in, int64_t nA, int64_t nB,
+                          int64_t n3, cudaStream_t s);
+
 // Path dispatch for the 3x3, stride-1 core (tensor-core kernel where the shape qualifies, else general).
 lrd_status_t conv3x3_fwd(const void* in, const void* G, void* out, int64_t B, int64_t H, int64_t W, int64_t ci,
                          int64_t co, lrd_dtype_t dt, int path, cudaStream_t s);

@@ -100,6 +100,29 @@ def test_tensor_core_path(geom, freeze):
     check_tucker(wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 500 + C), freeze)
 
 
+@pytest.mark.parametrize("geom", [(2, 14, 14, 256, 256, 96, 96), (2, 20, 14, 64, 64, 32, 32), (1, 5, 40, 16, 16, 16, 16), (1, 33, 3, 24, 40, 16, 16),
+                                  (3, 9, 11, 72, 200, 48, 64), (2, 4, 1, 16, 16, 16, 16), (2, 13, 30, 136, 256, 128, 128),
+                                  (1, 16, 16, 264, 88, 112, 80)])
+@pytest.mark.parametrize("freeze", MASKS)
+def test_whole_pass_in_one_launch(geom, freeze):
+    """Shapes the one-launch data passes take (ranks multiples of 16 up to 128, at most 256 output channels): tiles
+    of 7, 9, 1, 25 ... image rows with a ragged last tile, images 1 to 40 pixels wide, input channels off a multiple
+    of 64; the forward is then ONE launch, and the separate launches (forced through the unfused path) agree with
+    the oracle on the same inputs."""
+    B, H, W, C, S, r1, r2 = geom
+    case = wl.random_tucker_case(B, H, W, C, S, r1, r2, 3, "bf16", 600 + H + W)
+    desc = b.tucker2_desc(B, H, W, C, S, r1, r2, b.LRD_BF16)
+    X, A, G, Bm, bias = (dev(case[k], "bf16") for k in ("X", "A", "G", "Bm", "b"))
+    ws = workspace(b.lrd_tucker2_workspace_bytes(desc, b.LRD_TK_FREEZE_FACTORS, 0))
+    Y = torch.empty(B, H, W, S, dtype=torch.bfloat16, device="cuda")
+    Z1 = torch.empty(B, H, W, r1, dtype=torch.bfloat16, device="cuda")
+    n0 = b.lrd_launch_count()
+    b.lrd_tucker2_fwd(desc, X, A, G, Bm, bias, Y, Z1, None, b.LRD_TK_FREEZE_FACTORS, ws)
+    assert b.lrd_launch_count() - n0 == 1
+    check_tucker(case, freeze)
+    check_tucker(case, freeze, path=b.LRD_PATH_UNFUSED)
+
+
 @pytest.mark.parametrize("geom", [(2, 7, 7, 512, 512, 136, 136), (2, 7, 7, 512, 512, 256, 256), (1, 7, 7, 512, 512, 304, 248),
                                   (3, 7, 7, 512, 512, 312, 312)])
 @pytest.mark.parametrize("freeze", MASKS)

@@ -243,8 +243,11 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
  * unfrozen; lrd_linear_bwd_weights forms the unfrozen factor's gradients (dU = dY^T Z_save with dbias, dV = X^T dZ),
  * zero-fills the frozen one's buffers, and may run on another stream beside the next layer's data call.  When V is
  * unfrozen the weights call reads the dZ its layer's data call left in the SAME workspace: order it after that call
- * (same stream, or an event) and let nothing else use the workspace in between.  Together the two calls do exactly
- * what lrd_linear_bwd does (same kernels, same bits); arguments, layouts and errors as there. */
+ * (same stream, or an event) and let nothing else use the workspace in between.  Together the two calls do what
+ * lrd_linear_bwd does: dX has the same bits; the weight gradients agree within rounding, because a weights call,
+ * meant to run beside other launches, splits its reduction over the tokens into fewer, larger shares (blocks in
+ * clusters of 2, which find free SMs next to a running data call, instead of clusters of up to 8) and so adds the
+ * same products in a different grouping; repeated calls give identical bits.  Arguments, layouts and errors as there. */
 lrd_status_t lrd_linear_bwd_data(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
                                  lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
 lrd_status_t lrd_linear_bwd_weights(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,

@@ -36,6 +36,9 @@ struct GemmArgs {
     void* a_colsum = nullptr;  // optional [M]: sum over k of A(m, k) (the bias gradient when A is dY); only on the
                                // tensor-core path with both operands MN-major, see tc_gemm_colsum_ok()
     lrd_dtype_t dtype;         // storage type of A, B, C, bias
+    int max_cluster_split = 0; // split weight gradients: largest cluster to split the reduction over (0 = automatic).  A
+                               // launch meant to run BESIDE others asks for 2: clusters of 4 or 8 need that many free
+                               // SMs inside one GPC, which a chain kernel on 128 of the 148 SMs never leaves
 };
 
 // True when the CUDA call succeeded.  With the environment variable LRD_LOG_ERRORS set, a failure is also written to

@@ -582,7 +582,8 @@ struct SplitPlan {
 // B through one SM's memory port); all blocks together must not exceed what L2 delivers.  The
 // candidates are tile widths that the reduction buffers fit (<= 192) and cluster sizes that divide
 // the tile into slices of whole 16-byte groups.
-static SplitPlan pick_split(int64_t M, int64_t N, int64_t K, bool ones) {
+static SplitPlan pick_split(int64_t M, int64_t N, int64_t K, bool ones, int max_cluster = 0) {
+    const int top = max_cluster >= 2 && max_cluster < kMaxClusterSplits ? max_cluster : kMaxClusterSplits;
     const int64_t mt = (M + BM - 1) / BM, kb = (K + BK - 1) / BK;
     SplitPlan best{pick_bn(M, N, true), 1, 1};
     if (ones && best.bn > 192) best.bn = 192;
@@ -593,7 +594,7 @@ static SplitPlan pick_split(int64_t M, int64_t N, int64_t K, bool ones) {
         const int64_t nt = (N + bn - 1) / bn;
         if (nt * bn >= N + 64 && bn > 64) continue;              // a narrower width covers N with less waste
         const int64_t tiles = mt * nt;
-        for (int S = kMaxClusterSplits; S >= 2; --S) {
+        for (int S = top; S >= 2; --S) {
             if (bn % (8 * S)) continue;
             if (tiles > max_active_clusters(S) || S > kb) continue;    // one wave: a second wave would double the time
             const double per_block = (double)((kb + S - 1) / S) * (A_STAGE_BYTES + bn * BK * 2.0);
@@ -610,8 +611,9 @@ int tc_pick_splits(int64_t M, int64_t N, int64_t K) { return pick_split(M, N, K,
 // fp32 partial tiles [splits][M][ldp], then (for the optional column sums) [splits][M]; nothing for a cluster split
 size_t tc_split_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     size_t need = 0;
-    for (int ones = 0; ones < 2; ++ones) {
-        const int s = pick_split(M, N, K, ones != 0).global;
+    for (int v = 0; v < 4; ++v) {                    // with and without the column sums, for either cluster limit
+        const int ones = v & 1;
+        const int s = pick_split(M, N, K, ones != 0, (v & 2) ? 2 : 0).global;
         const size_t n = s > 1 ? align_up((size_t)s * M * ((N + 3) / 4 * 4) * sizeof(float), 256) + align_up((size_t)s * M * sizeof(float), 256) : 0;
         need = need > n ? need : n;
     }
@@ -630,7 +632,7 @@ lrd_status_t tc_gemm(const GemmArgs& g, bool allow_split, float* partials, size_
     if (!allow_split && !ones) return tc_gemm_persistent(g, stream);   // data products: the persistent kernel
     int splits = 1, cluster = 1, bn;
     if (allow_split) {
-        const SplitPlan sp = pick_split(g.M, g.N, g.K, ones);
+        const SplitPlan sp = pick_split(g.M, g.N, g.K, ones, g.max_cluster_split);
         bn = sp.bn; cluster = sp.cluster; splits = sp.global;
     } else {
         bn = pick_bn(g.M, g.N, false);

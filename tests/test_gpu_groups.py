@@ -58,14 +58,15 @@ class Group:
                     continue
                 got = self.out[name][li]
                 assert rel_err(got, ref[name]) <= TOL["bf16"], (li, name)
-                # A group changes where and beside what a layer runs.  The intermediate and the weight gradients are
-                # summed in the same order as in a single-layer call (same bits); the second product of a chain walks
-                # over the rank in an order that depends on the cluster size, so Y and dX agree to rounding only.
+                # A group changes where and beside what a layer runs.  The intermediate has the bits of a single-layer
+                # call; the second product of a chain walks over the rank in an order that depends on the cluster size,
+                # and the weight gradients of a group reduce over the tokens in fewer, larger shares, so Y, dX and
+                # the weight gradients agree to rounding only.
                 if one is not None and one[name] is not None:
-                    if name in ("Y", "dX"):
-                        assert rel_err(got, host(one[name])) <= 2.0 ** -7, (li, name)
-                    else:
+                    if name == "Z":
                         assert torch.equal(got, one[name]), (li, name)
+                    else:
+                        assert rel_err(got, host(one[name])) <= 2.0 ** -7, (li, name)
 
 
 QKV = [(520, 264, 264, 64)] * 3

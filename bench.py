@@ -622,6 +622,8 @@ def run_other(args):
                           "dW": acts[name].setdefault("dW", torch.empty(N, K, dtype=bf, device="cuda")),
                           "ddesc": b.linear_desc(M, K, N, 0, b.LRD_BF16)})
                 L["wsd"] = acts[name].setdefault("wsd", torch.empty(max(b.lrd_dense_workspace_bytes(L["ddesc"], 1), 256), dtype=torch.uint8, device="cuda"))
+                if not name.startswith(("attn_q", "attn_k", "attn_v")):
+                    L["ws"] = torch.empty_like(acts[name]["ws"])
                 layers.append(L)
             blocks.append(layers)
 
@@ -655,8 +657,23 @@ def run_other(args):
             for bi, layers in reversed(list(enumerate(blocks))):
                 ss = (s + bi) % S
                 for L in reversed(layers[3:]):
-                    one_bwd(L, ss, f)
+                    if args.wgrad != "beside":
+                        one_bwd(L, ss, f)
+                        continue
+                    # the weight gradients on a second stream beside the next layer's data pass (each layer of each
+                    # block has its own workspace: the weights call reads the dZ its data call left there)
+                    st = L["sets"][ss]
+                    cur = torch.cuda.current_stream()
+                    b.lrd_linear_bwd_data(L["desc"], st["dY"], L["V"], L["U"], st["dX"], f, L["ws"])
+                    c4_w.wait_stream(cur)
+                    with torch.cuda.stream(c4_w):
+                        b.lrd_linear_bwd_weights(L["desc"], st["dY"], None if f == 2 else st["X"], None if f == 1 else st["Z"],
+                                                 None if f == 1 else L["dU"], None if f == 2 else L["dV"], None if f == 1 else L["db"], f, L["ws"])
                 g_call(layers[:3], ss, f, False)
+            if args.wgrad == "beside":
+                torch.cuda.current_stream().wait_stream(c4_w)
+
+        c4_w = torch.cuda.Stream()
 
         def dense_stack(s):
             for bi, layers in enumerate(blocks):

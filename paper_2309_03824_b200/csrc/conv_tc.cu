@@ -47,7 +47,7 @@ struct ConvParams {
     const __nv_bfloat16* bias2;   // [n2] or nullptr
 };
 
-// grid: (ceil(n_total / 128), tiles_per_img, B); fused: n_total <= 128, so gridDim.x = 1
+// grid: (ceil(n_total / 128), tiles_per_img, B); fused: gridDim.x = 1 and the block walks over the (one or two) column tiles
 template <bool DGRAD, bool FUSE>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ CUtensorMap tmG,
@@ -60,7 +60,9 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const AbortCtx ab{&abort_flag, p.timeout_flag};
     const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
-    const int n0 = blockIdx.x * 128, h0 = blockIdx.y * p.bh, img = blockIdx.z;
+    const int h0 = blockIdx.y * p.bh, img = blockIdx.z;
+    // 128-column tiles of the core's result: one per block (gridDim.x), or, fused, all of them (up to two) in this block
+    const int n_tiles = FUSE ? (p.n_total + 127) / 128 : 1;
     const int nkc = (p.ka + 63) / 64;                  // 64-channel blocks per tap
     const int iters = 9 * nkc;
     const uint32_t a_bytes = (uint32_t)(p.bh * p.W) * 128u;
@@ -93,19 +95,22 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
     // overlaps the tail of the previous kernel in the stream; global memory is first touched below this line
     griddep_launch_dependents();
     griddep_wait();
-    // fused: once the core's MMAs are done the ring is dead; it then holds [T: 2 atoms of 128 rows x 64 columns |
-    // Q: one [256 rows x 64 k] tile per 64 columns of the core's result]
-    const uint32_t t_base = smem_base, q_base = smem_base + 2 * kTile;
+    // fused: once the core's MMAs are done the ring is dead; it then holds [T: one atom of 128 rows x 64 columns per 64
+    // columns of the core's result | Q: one [256 rows x 64 k] tile per 64 columns of the core's result]
     const int nq = (p.n_total + 63) / 64;
+    const uint32_t t_base = smem_base, q_base = smem_base + (uint32_t)nq * kTile;
 
     if (warp == 0) {
         // TMA producer: the whole warp runs the loop, one elected lane issues
         int s = 0;
         uint32_t ph = 1;
+        bool go = true;
+        for (int nt = 0; nt < n_tiles && go; ++nt)
         for (int it = 0; it < iters; ++it) {
+            const int n0 = FUSE ? nt * 128 : (int)blockIdx.x * 128;
             const int tap = it / nkc, cb = it % nkc;
             const int kh = tap / 3, kw = tap % 3;
-            if (!mbar_wait_uniform(smem_u32(&empty_bar[s]), ph, ab)) break;
+            if (!mbar_wait_uniform(smem_u32(&empty_bar[s]), ph, ab)) { go = false; break; }
             const uint32_t fb = smem_u32(&full_bar[s]);
             const uint32_t a_dst = smem_base + s * kStageBytes, b_dst = a_dst + kTile;
             if (elect_one()) {
@@ -137,18 +142,20 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
         int s = 0;
         uint32_t ph = 0;
         bool ok = true;
+        for (int nt = 0; nt < n_tiles && ok; ++nt)
         for (int it = 0; it < iters; ++it) {
             ok = mbar_wait_uniform(smem_u32(&full_bar[s]), ph, ab);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a_src = smem_base + s * kStageBytes, b_src = a_src + kTile;
+            const uint32_t acc = tmem_base + (uint32_t)nt * 128u;
             const int nks = min(4, (p.ka - (it % nkc) * 64 + 15) / 16);      // 16-channel steps past ka hold zeros: not issued
             if (elect_one()) {
                 const uint64_t ad0 = smem_desc_sw128(a_src, 0, 1024);
                 const uint64_t bd0 = DGRAD ? smem_desc_sw128(b_src, 8192, 1024) : smem_desc_sw128(b_src, 0, 1024);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)                               // the k-step moves the start address only
-                    if (kk < nks) mma_bf16_ss(tmem_base, ad0 + 2u * kk, bd0 + (DGRAD ? 128u : 2u) * kk, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    if (kk < nks) mma_bf16_ss(acc, ad0 + 2u * kk, bd0 + (DGRAD ? 128u : 2u) * kk, idesc, (it > 0 || kk > 0) ? 1u : 0u);
                 mma_commit(smem_u32(&empty_bar[s]));
             }
             __syncwarp();
@@ -181,8 +188,9 @@ conv_kernel(const __grid_constant__ CUtensorMap tmImg, const __grid_constant__ C
         const bool row_ok = row < p.bh * p.W && h0 + row / p.W < p.H;
         if (ready) {
             __nv_bfloat16* dst_row = p.out + ((int64_t)(img * p.H + h0) * p.W + row) * p.n_total;
+            const int n0 = FUSE ? 0 : (int)blockIdx.x * 128;
 #pragma unroll 1
-            for (int cchunk = 0; cchunk < 4; ++cchunk) {
+            for (int cchunk = 0; cchunk < 4 * n_tiles; ++cchunk) {
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + cchunk * 32, v);
                 tmem_ld_wait();
@@ -525,7 +533,7 @@ bool tc_conv_chain_eligible(bool dgrad, int64_t B, int64_t H, int64_t W, int64_t
                             const void* img, const void* G, const void* Q, const void* out2, const void* core_out) {
     const int64_t n1 = dgrad ? ci : co;                  // channels of the core's result = reduction of the 1x1 product
     if (!tc_conv_eligible(B, H, W, ci, co, dt, img, G, Q)) return false;
-    if (n1 > 128 || n1 % 16 || n2 < 8 || n2 > 256 || n2 % 8) return false;
+    if (n1 > 256 || n1 % 16 || n2 < 8 || n2 > 256 || n2 % 8) return false;
     return a16(out2) && (!core_out || a16(core_out));
 }
 

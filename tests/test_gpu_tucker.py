@@ -93,7 +93,8 @@ def test_geometries_outside_the_supported_set_are_refused():
 
 
 @pytest.mark.parametrize("geom", [(4, 14, 14, 64, 72, 32, 40), (2, 9, 11, 128, 136, 96, 104), (5, 14, 14, 256, 256, 96, 96),
-                                  (3, 10, 12, 72, 200, 48, 64), (2, 7, 9, 40, 24, 16, 16), (1, 14, 14, 256, 248, 128, 112)])
+                                  (3, 10, 12, 72, 200, 48, 64), (2, 7, 9, 40, 24, 16, 16), (1, 14, 14, 256, 248, 128, 112),
+                                  (2, 9, 11, 256, 256, 144, 160), (1, 14, 14, 256, 256, 256, 256), (2, 6, 50, 64, 64, 32, 48)])
 @pytest.mark.parametrize("freeze", MASKS)
 def test_tensor_core_path(geom, freeze):
     B, H, W, C, S, r1, r2 = geom

@@ -198,6 +198,12 @@ lrd_status_t lrd_tucker2_overlap(int on);
  * LRD_OK, LRD_ERR_TIMEOUT, or LRD_ERR_CUDA if the synchronisation itself failed. */
 lrd_status_t lrd_check_device_status(void);
 
+/* Debug mode (no counterpart in the paper).  With the environment variable LRD_DEBUG set (to anything but 0) when the
+ * library is loaded, every compute entry point below waits for the work it has enqueued and returns what went wrong
+ * in it: LRD_ERR_CUDA for a launch or execution error, LRD_ERR_TIMEOUT for a bounded device wait that ran out (the
+ * flag is cleared, as by lrd_check_device_status).  A call whose stream is being captured is left alone.  Off by
+ * default, where the library never synchronises and errors surface at lrd_check_device_status(). */
+
 /* Self-test of the bounded device-side wait (no counterpart in the paper): enqueues one small block that waits,
  * through the same routine and with the same limit as every pipeline wait of the library's kernels, on a barrier
  * nothing ever arrives at.  The wait runs out after a second or so, raises the timeout flag and the block

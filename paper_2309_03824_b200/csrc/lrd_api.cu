@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
 
 #include "chain.cuh"
 #include "common.cuh"
@@ -478,7 +479,7 @@ static lrd_status_t linear_fwd_on(const lrd_linear_desc_t* desc, const void* X, 
     return run_gemm(gemm(L.M, L.N, L.r, Z, ldz, false, U, L.ldu, false, Y, L.ldy, bias, L.dt), false, nullptr, 0, s);
 }
 
-lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
+static lrd_status_t lrd_linear_fwd_impl(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
                             const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze, void* workspace,
                             size_t workspace_bytes, void* cuda_stream) {
     return linear_fwd_on(desc, X, V, U, bias, Y, Z_save, freeze, workspace, workspace_bytes, (cudaStream_t)cuda_stream, 0);
@@ -589,27 +590,27 @@ static lrd_status_t linear_bwd_on(const lrd_linear_desc_t* desc, const void* dY,
     return LRD_OK;
 }
 
-lrd_status_t lrd_linear_bwd_data(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
+static lrd_status_t lrd_linear_bwd_data_impl(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
                                  lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return linear_bwd_on(desc, dY, nullptr, V, U, nullptr, dX, nullptr, nullptr, nullptr, freeze, workspace, workspace_bytes,
                          (cudaStream_t)cuda_stream, nullptr, nullptr, 0, false, 1);
 }
 
-lrd_status_t lrd_linear_bwd_weights(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,
+static lrd_status_t lrd_linear_bwd_weights_impl(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,
                                     void* dV, void* dbias, lrd_freeze_t freeze, void* workspace, size_t workspace_bytes,
                                     void* cuda_stream) {
     return linear_bwd_on(desc, dY, X, nullptr, nullptr, Z_save, nullptr, dU, dV, dbias, freeze, workspace, workspace_bytes,
                          (cudaStream_t)cuda_stream, nullptr, nullptr, 0, false, 2);
 }
 
-lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+static lrd_status_t lrd_linear_bwd_impl(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
                             const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                             lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return linear_bwd_on(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, workspace_bytes,
                          (cudaStream_t)cuda_stream, nullptr, nullptr, 0);
 }
 
-lrd_status_t lrd_linear_bwd_accumulate(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+static lrd_status_t lrd_linear_bwd_accumulate_impl(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
                                        const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
                                        lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     Linear L;
@@ -645,7 +646,7 @@ lrd_status_t lrd_linear_bwd_accumulate(const lrd_linear_desc_t* desc, const void
 // ---- groups of independent layers -------------------------------------------------------------------
 // Layer 0 of a group runs on the caller's stream, layer i on side stream i - 1; the dU products of a backward
 // group use the auxiliary set.
-lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
+static lrd_status_t lrd_linear_group_fwd_impl(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
                                   const void* const* U, const void* const* bias, void* const* Y, void* const* Z_save,
                                   lrd_freeze_t freeze, void* const* workspace, const size_t* workspace_bytes,
                                   void* cuda_stream) {
@@ -684,7 +685,7 @@ lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const v
     return st;
 }
 
-lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const void* const* dY, const void* const* X,
+static lrd_status_t lrd_linear_group_bwd_impl(int n, const lrd_linear_desc_t* descs, const void* const* dY, const void* const* X,
                                   const void* const* V, const void* const* U, const void* const* Z_save, void* const* dX,
                                   void* const* dU, void* const* dV, void* const* dbias, lrd_freeze_t freeze,
                                   void* const* workspace, const size_t* workspace_bytes, void* cuda_stream) {
@@ -740,7 +741,7 @@ lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const v
     return st;
 }
 
-lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const void* W, const void* bias, void* Y,
+static lrd_status_t lrd_dense_fwd_impl(const lrd_linear_desc_t* desc, const void* X, const void* W, const void* bias, void* Y,
                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
     Linear L;
     LRD_TRY(parse_linear(desc, &L, true));
@@ -753,7 +754,7 @@ lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const v
                     (cudaStream_t)cuda_stream);
 }
 
-lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* W, void* dX,
+static lrd_status_t lrd_dense_bwd_impl(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* W, void* dX,
                            void* dW, void* dbias, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     Linear L;
     LRD_TRY(parse_linear(desc, &L, true));
@@ -793,7 +794,7 @@ size_t lrd_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C, i
     return align_up(dtype == LRD_BF16 ? tc_conv_filter_scratch_bytes(B, H, W, C, S) : 0, 256) + 256;
 }
 
-lrd_status_t lrd_conv3x3_fwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* X, const void* Wk,
+static lrd_status_t lrd_conv3x3_fwd_impl(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* X, const void* Wk,
                              void* Y, void* cuda_stream) {
     LRD_TRY(conv3x3_check(B, H, W, C, S, dtype));
     if (!X || !Wk || !Y) return LRD_ERR_INVALID_ARG;
@@ -804,7 +805,7 @@ lrd_status_t lrd_conv3x3_fwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t
     return conv3x3_fwd(X, Wk, Y, B, H, W, C, S, (lrd_dtype_t)dtype, g_path.load(), (cudaStream_t)cuda_stream);
 }
 
-lrd_status_t lrd_conv3x3_bwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* dY, const void* X,
+static lrd_status_t lrd_conv3x3_bwd_impl(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* dY, const void* X,
                              const void* Wk, void* dX, void* dW, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     LRD_TRY(conv3x3_check(B, H, W, C, S, dtype));
     if (!dY || !X || !Wk || !dW) return LRD_ERR_INVALID_ARG;
@@ -822,7 +823,7 @@ size_t lrd_tucker2_workspace_bytes(const lrd_tucker2_desc_t* desc, lrd_tucker_fr
     return tucker2_workspace_bytes(desc, freeze, is_bwd);
 }
 
-lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, const void* A, const void* G,
+static lrd_status_t lrd_tucker2_fwd_impl(const lrd_tucker2_desc_t* desc, const void* X, const void* A, const void* G,
                              const void* Bm, const void* bias, void* Y, void* Z1_save, void* Z2_save,
                              lrd_tucker_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     LRD_TRY(tucker2_check(desc, freeze));
@@ -837,7 +838,7 @@ lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, cons
                        g_path.load(), (cudaStream_t)cuda_stream);
 }
 
-lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, const void* X, const void* A,
+static lrd_status_t lrd_tucker2_bwd_impl(const lrd_tucker2_desc_t* desc, const void* dY, const void* X, const void* A,
                              const void* G, const void* Bm, const void* Z1_save, const void* Z2_save, void* dX,
                              void* dA, void* dG, void* dB, void* dbias, lrd_tucker_freeze_t freeze, void* workspace,
                              size_t workspace_bytes, void* cuda_stream) {
@@ -851,6 +852,103 @@ lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, con
     LRD_TRY(check_arch());
     return tucker2_bwd(desc, dY, X, A, G, Bm, Z1_save, Z2_save, dX, dA, dG, dB, dbias, freeze, workspace,
                        workspace_bytes, g_path.load(), (cudaStream_t)cuda_stream);
+}
+
+
+// ---- debug mode ---------------------------------------------------------------------------------------------------
+// With the environment variable LRD_DEBUG set (to anything but 0), every compute entry point waits for the work it has
+// enqueued and reports what went wrong in it -- LRD_ERR_CUDA for a launch or execution error, LRD_ERR_TIMEOUT for a
+// bounded device wait that ran out -- instead of leaving both to the next lrd_check_device_status().  A call made
+// while its stream is being captured is left alone.  Off by default: the library otherwise never synchronises.
+static bool debug_on() {
+    static const bool on = [] { const char* e = getenv("LRD_DEBUG"); return e && *e && strcmp(e, "0") != 0; }();
+    return on;
+}
+static lrd_status_t debug_checked(lrd_status_t st, void* cuda_stream) {
+    if (st != LRD_OK || !debug_on()) return st;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing((cudaStream_t)cuda_stream, &cap) != cudaSuccess) { cudaGetLastError(); return st; }
+    if (cap != cudaStreamCaptureStatusNone) return st;
+    if (!cuda_ok(cudaStreamSynchronize((cudaStream_t)cuda_stream), "cudaStreamSynchronize(LRD_DEBUG)")) return LRD_ERR_CUDA;
+    bool raised = false;
+    if (read_and_clear_device_timeout(&raised) != LRD_OK) return LRD_ERR_CUDA;
+    return raised ? LRD_ERR_TIMEOUT : LRD_OK;
+}
+
+lrd_status_t lrd_linear_fwd(const lrd_linear_desc_t* desc, const void* X, const void* V, const void* U,
+                            const void* bias, void* Y, void* Z_save, lrd_freeze_t freeze, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_linear_fwd_impl(desc, X, V, U, bias, Y, Z_save, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_linear_bwd_data(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
+                                 lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_linear_bwd_data_impl(desc, dY, V, U, dX, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_linear_bwd_weights(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,
+                                    void* dV, void* dbias, lrd_freeze_t freeze, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+    return debug_checked(lrd_linear_bwd_weights_impl(desc, dY, X, Z_save, dU, dV, dbias, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                            const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                            lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_linear_bwd_impl(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_linear_bwd_accumulate(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* V,
+                                       const void* U, const void* Z_save, void* dX, void* dU, void* dV, void* dbias,
+                                       lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_linear_bwd_accumulate_impl(desc, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_linear_group_fwd(int n, const lrd_linear_desc_t* descs, const void* const* X, const void* const* V,
+                                  const void* const* U, const void* const* bias, void* const* Y, void* const* Z_save,
+                                  lrd_freeze_t freeze, void* const* workspace, const size_t* workspace_bytes,
+                                  void* cuda_stream) {
+    return debug_checked(lrd_linear_group_fwd_impl(n, descs, X, V, U, bias, Y, Z_save, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_linear_group_bwd(int n, const lrd_linear_desc_t* descs, const void* const* dY, const void* const* X,
+                                  const void* const* V, const void* const* U, const void* const* Z_save, void* const* dX,
+                                  void* const* dU, void* const* dV, void* const* dbias, lrd_freeze_t freeze,
+                                  void* const* workspace, const size_t* workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_linear_group_bwd_impl(n, descs, dY, X, V, U, Z_save, dX, dU, dV, dbias, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_dense_fwd(const lrd_linear_desc_t* desc, const void* X, const void* W, const void* bias, void* Y,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_dense_fwd_impl(desc, X, W, bias, Y, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_dense_bwd(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* W, void* dX,
+                           void* dW, void* dbias, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_dense_bwd_impl(desc, dY, X, W, dX, dW, dbias, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_conv3x3_fwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* X, const void* Wk,
+                             void* Y, void* cuda_stream) {
+    return debug_checked(lrd_conv3x3_fwd_impl(B, H, W, C, S, dtype, X, Wk, Y, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_conv3x3_bwd(int64_t B, int64_t H, int64_t W, int64_t C, int64_t S, int dtype, const void* dY, const void* X,
+                             const void* Wk, void* dX, void* dW, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_conv3x3_bwd_impl(B, H, W, C, S, dtype, dY, X, Wk, dX, dW, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_tucker2_fwd(const lrd_tucker2_desc_t* desc, const void* X, const void* A, const void* G,
+                             const void* Bm, const void* bias, void* Y, void* Z1_save, void* Z2_save,
+                             lrd_tucker_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_tucker2_fwd_impl(desc, X, A, G, Bm, bias, Y, Z1_save, Z2_save, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
+}
+
+lrd_status_t lrd_tucker2_bwd(const lrd_tucker2_desc_t* desc, const void* dY, const void* X, const void* A,
+                             const void* G, const void* Bm, const void* Z1_save, const void* Z2_save, void* dX,
+                             void* dA, void* dG, void* dB, void* dbias, lrd_tucker_freeze_t freeze, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    return debug_checked(lrd_tucker2_bwd_impl(desc, dY, X, A, G, Bm, Z1_save, Z2_save, dX, dA, dG, dB, dbias, freeze, workspace, workspace_bytes, cuda_stream), cuda_stream);
 }
 
 }  // extern "C"

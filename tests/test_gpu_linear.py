@@ -144,6 +144,36 @@ def test_a_bounded_wait_that_runs_out_is_reported_once():
     check_linear(wl.random_factor_case(300, 200, 136, 64, "bf16", 370), b.LRD_FREEZE_NONE)
 
 
+def test_debug_mode_reports_at_the_call():
+    """LRD_DEBUG=1: an entry point waits for its own work, so a device wait that ran out before it is reported (and
+    cleared) by the next compute call itself, and a clean call returns LRD_OK with its results complete."""
+    import os
+    import subprocess
+    import sys
+    code = """
+import torch
+from paper_2309_03824_b200 import binding as b, workloads as wl
+from helpers import check_linear
+check_linear(wl.random_factor_case(300, 200, 136, 64, "bf16", 371), b.LRD_FREEZE_NONE)
+b.lrd_selftest_wait_timeout()
+case = wl.random_factor_case(300, 200, 136, 64, "bf16", 372)
+bf = torch.bfloat16
+X, V, U, bias = (torch.from_numpy(case[k]).to("cuda", bf) for k in ("X", "V", "U", "b"))
+desc = b.linear_desc(300, 200, 136, 64, b.LRD_BF16)
+Y = torch.empty(300, 136, dtype=bf, device="cuda")
+ws = torch.empty(max(b.lrd_linear_workspace_bytes(desc, 1, 0), 256), dtype=torch.uint8, device="cuda")
+st = b.lrd_linear_fwd(desc, X, V, U, bias, Y, None, b.LRD_FREEZE_U, ws, check=False)
+assert st == b.LRD_ERR_TIMEOUT, st
+assert b.lrd_linear_fwd(desc, X, V, U, bias, Y, None, b.LRD_FREEZE_U, ws, check=False) == b.LRD_OK
+assert b.lrd_check_device_status() == b.LRD_OK
+print("debug mode ok")
+"""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, LRD_DEBUG="1", PYTHONPATH=os.pathsep.join([root, os.path.join(root, "tests")]))
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and "debug mode ok" in out.stdout, out.stderr[-2000:]
+
+
 def _svd_factors(W, r):
     Uf, s, Vt = np.linalg.svd(W, full_matrices=False)     # input construction only
     root = np.sqrt(s[:r])

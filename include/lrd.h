@@ -250,10 +250,11 @@ lrd_status_t lrd_linear_bwd(const lrd_linear_desc_t* desc, const void* dY, const
  * zero-fills the frozen one's buffers, and may run on another stream beside the next layer's data call.  When V is
  * unfrozen the weights call reads the dZ its layer's data call left in the SAME workspace: order it after that call
  * (same stream, or an event) and let nothing else use the workspace in between.  Together the two calls do what
- * lrd_linear_bwd does: dX has the same bits; the weight gradients agree within rounding, because a weights call,
- * meant to run beside other launches, splits its reduction over the tokens into fewer, larger shares (blocks in
- * clusters of 2, which find free SMs next to a running data call, instead of clusters of up to 8) and so adds the
- * same products in a different grouping; repeated calls give identical bits.  Arguments, layouts and errors as there. */
+ * lrd_linear_bwd does, with launch shapes chosen to leave room for each other: the data call takes the fused chain on
+ * pairs of SMs where the shape allows (fewer blocks), the weights call splits its reduction over the tokens into fewer,
+ * larger shares (blocks in clusters of 2, which find free SMs next to a running data call, instead of clusters of up
+ * to 8).  The same products are therefore added in a different grouping: results agree with lrd_linear_bwd within
+ * rounding; repeated calls give identical bits.  Arguments, layouts and errors as there. */
 lrd_status_t lrd_linear_bwd_data(const lrd_linear_desc_t* desc, const void* dY, const void* V, const void* U, void* dX,
                                  lrd_freeze_t freeze, void* workspace, size_t workspace_bytes, void* cuda_stream);
 lrd_status_t lrd_linear_bwd_weights(const lrd_linear_desc_t* desc, const void* dY, const void* X, const void* Z_save, void* dU,

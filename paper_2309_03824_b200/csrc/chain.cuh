@@ -35,6 +35,7 @@ constexpr int kChainMaxLayers = 4;
 void chain_pair_tuning(int S, int G1, int BN2);
 bool chain_pair_eligible(const ChainArgs* layers, int n);
 bool chain_pair_preferred(const ChainArgs* layers, int n);
+bool chain_pair_roomy(const ChainArgs* layers, int n);
 lrd_status_t chain_pair_launch(const ChainArgs* layers, int n, cudaStream_t stream);
 
 }  // namespace lrd

@@ -581,6 +581,14 @@ bool chain_pair_preferred(const ChainArgs* layers, int n) {
     return n > 1 || a.K1 >= 2 * a.N2 || (a.r > 384 && !chain_preferred(a)) || (a.r >= 384 && (a.M + 127) / 128 > 37);
 }
 
+// Eligible, with at least three weight tiles of the second product in flight: the form to take where the launch should
+// leave SMs free for others (16 clusters of 6 or fewer blocks against 32 clusters of 4).
+bool chain_pair_roomy(const ChainArgs* layers, int n) {
+    if (!chain_pair_eligible(layers, n)) return false;
+    Plan pl;
+    return make_plan(layers[0], n, &pl) && pl.NS2 >= 3;
+}
+
 lrd_status_t chain_pair_launch(const ChainArgs* layers, int n, cudaStream_t stream) {
     if (!chain_pair_eligible(layers, n)) return LRD_ERR_UNSUPPORTED;
     const ChainArgs& a = layers[0];
